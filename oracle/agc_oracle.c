@@ -1,0 +1,349 @@
+/*
+ * CPU oracle for the per-round path of joint approximate gradient coding and
+ * quantisation: encode (Sec. II-A, f_i = sum_j a_ij g_j), stochastic
+ * quantisation (Sec. II-B, Eq. quant_def / Eq. rv_quant, bucket-wise variant),
+ * bit packing, and the master's straggler-masked weighted decode
+ * (Sec. II-A, g_hat = sum_i I_i w_i q_i) with the update of Eq. update_param.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE. It is plain, slow, single-threaded and
+ * written to be checked against the paper by eye. Nothing in the product path
+ * may call it; it shares no code with the CUDA kernels.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC (see build.py).
+ * Every fp32 operation below is a single IEEE-754 binary32 operation with
+ * round-to-nearest-even; fmaf() is the correctly rounded fused multiply-add.
+ *
+ * Notation: n workers, k partitions, d coordinates, b_i bits of worker i,
+ * L_i = 2^(b_i-1) - 1 magnitude levels (the paper's s_i), B bucket size.
+ *
+ * Wire format (the paper only counts bits; the layout is this build's):
+ *   - coordinates are grouped in pack blocks of 512; inside a block the
+ *     coordinate with offset o = 128*c + 4*l + e (c<4, l<32, e<4) sits at
+ *     stream position 16*l + 4*c + e;
+ *   - worker i's message is a little-endian bit stream over 32-bit words with
+ *     b_i bits per stream position, padded to whole blocks (16*b_i words each);
+ *   - messages are concatenated in worker order;
+ *   - scales[i*nb + beta] is the l2 norm of bucket beta of worker i.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define AGC_BLOCK 512
+#define AGC_FRAC_BITS 15
+
+/* status bits reported by the encoder */
+#define AGC_ORACLE_STATUS_NONFINITE 1u  /* a bucket had a NaN/Inf sum of squares */
+#define AGC_ORACLE_STATUS_RANGE 2u      /* a code left [0, 2L]: must never happen  */
+
+/* ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers:
+ * as easy as 1, 2, 3", SC'11). The paper asks only for "lightweight shared
+ * random seeds" (Sec. II-B); a counter-based generator makes every draw a pure
+ * function of (seed, round, worker, stream position). ---- */
+void agc_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* 15-bit uniform integer for stream position pos of worker i in a round.
+ * One Philox block serves 8 consecutive stream positions: two per output word,
+ * the even one from the low 15 bits, the odd one from the high 15 bits. */
+uint32_t agc_oracle_uniform15(uint64_t seed, uint64_t round, uint32_t worker, uint64_t pos)
+{
+    uint32_t ctr[4] = { (uint32_t)(pos >> 3), worker, (uint32_t)round, (uint32_t)(round >> 32) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    agc_oracle_philox4x32_10(ctr, key, out);
+    uint32_t word = out[(pos & 7) >> 1];
+    return (pos & 1) ? (word >> 17) : (word & 0x7FFFu);
+}
+
+/* stream position of coordinate offset o (0..511) inside its pack block */
+static inline int stream_pos_in_block(int o)
+{
+    int c = o >> 7, l = (o >> 2) & 31, e = o & 3;
+    return 16 * l + 4 * c + e;
+}
+
+int64_t agc_oracle_stream_position(int64_t m)
+{
+    return (m / AGC_BLOCK) * AGC_BLOCK + stream_pos_in_block((int)(m % AGC_BLOCK));
+}
+
+/* per-worker quantiser constants.
+ * b >= 2 (the paper's case): grid {-L..L}/L, offset-binary code = level + L.
+ * b == 1 (extension outside the paper, which requires z_i >= 2): the two-point
+ *        unbiased quantiser {-S, +S} with P(+S) = (1 + x/S)/2. */
+static float enc_scale(int b)  { return b >= 2 ? (float)(((1 << (b - 1)) - 1) << AGC_FRAC_BITS) : 16384.0f; }
+static uint32_t enc_offset(int b) { return b >= 2 ? (uint32_t)(((1 << (b - 1)) - 1) << AGC_FRAC_BITS) : 16384u; }
+static float dec_offset(int b) { return b >= 2 ? (float)((1 << (b - 1)) - 1) : 0.5f; }
+static float dec_step(int b)   { return b >= 2 ? (float)(1.0 / (double)((1 << (b - 1)) - 1)) : 2.0f; }
+static uint32_t zero_code(int b) { return b >= 2 ? (uint32_t)((1 << (b - 1)) - 1) : 0u; }
+
+static inline uint32_t f2u(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+/* Eq. rv_quant for one coordinate. inv = enc_scale(b)/S. With y = L*x/S the
+ * paper's rule (level floor(y) or floor(y)+1, the latter w.p. y - floor(y))
+ * is level = floor(y + r) for r uniform in [0,1); it also holds for negative y,
+ * so the sign needs no separate treatment. r = u/2^15, and the sum is formed
+ * in fixed point with 15 fractional bits inside the mantissa of a float in
+ * [2^23, 2^24): one correctly rounded fma gives round(x*inv) + offset + u.
+ * Returns the offset-binary code level + L (b >= 2), or the bit of the
+ * two-point quantiser (b == 1), before masking to b bits. */
+uint32_t agc_oracle_quantize_one(float x, float inv, int b, uint32_t u)
+{
+    float addend = (float)(8388608u + enc_offset(b) + u); /* exact: an integer below 2^24 */
+    float tq = fmaf(x, inv, addend);
+    uint32_t fixed = f2u(tq) - 0x4B000000u;
+    return fixed >> AGC_FRAC_BITS;
+}
+
+/* the fp32 reciprocal scale the encoder multiplies by: enc_scale(b) / S */
+float agc_oracle_inv_scale(float S, int b) { return enc_scale(b) / S; }
+
+/* dequantised value of one code: (w*S*step) * (code - offset) */
+float agc_oracle_dequantize_one(uint32_t code, float S, int b)
+{
+    return (S * dec_step(b)) * ((float)code - dec_offset(b));
+}
+
+/* l2 norm of one bucket (Eq. quant_def's ||x||_2 restricted to the bucket).
+ * Summation order (the paper is silent): view the bucket as rows of 128;
+ * column sums by fused multiply-add over the rows in order, then a pairwise
+ * tree over the 128 column sums in index order. Returns the sum of squares. */
+static float bucket_sumsq(const float *x, int B)
+{
+    float p[128];
+    for (int c = 0; c < 128; ++c) p[c] = 0.0f;
+    for (int r = 0; r < B / 128; ++r)
+        for (int c = 0; c < 128; ++c)
+            p[c] = fmaf(x[r * 128 + c], x[r * 128 + c], p[c]);
+    for (int width = 64; width >= 1; width >>= 1)
+        for (int t = 0; t < width; ++t)
+            p[t] = p[2 * t] + p[2 * t + 1];
+    return p[0];
+}
+
+/*
+ * Encode + quantise + pack ONE pack block (512 coordinates) for every worker.
+ *   q          block index (stream positions 512q .. 512q+511)
+ *   Gblk       k x 512 row-major slice of the partial gradients, coordinates
+ *              beyond d already set to +0
+ *   codes_blk  out: for worker i, 16*b_i words starting at word 16*sum_{i'<i} b_i'
+ *   scales_blk out: n x (512/B), bucket-in-block minor
+ *   x_out      optional out: n x 512 coded values f_i before quantisation
+ * Returns status bits.
+ */
+uint32_t agc_oracle_encode_block(int n, const int32_t *row_ptr, const int32_t *col_idx,
+                                 const float *a, const uint8_t *bits, int B, uint64_t seed,
+                                 uint64_t round, int64_t q, const float *Gblk,
+                                 uint32_t *codes_blk, float *scales_blk, float *x_out)
+{
+    uint32_t status = 0;
+    int word_base = 0;
+    for (int i = 0; i < n; ++i) {
+        const int b = bits[i];
+        float x[AGC_BLOCK];
+        /* Sec. II-A: f_i = sum_{j in supp(i)} a_ij g_j, ascending j, fp32 fma chain */
+        for (int o = 0; o < AGC_BLOCK; ++o) {
+            float acc = 0.0f;
+            for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                acc = fmaf(a[e], Gblk[(int64_t)col_idx[e] * AGC_BLOCK + o], acc);
+            x[o] = acc;
+        }
+        if (x_out) memcpy(x_out + (int64_t)i * AGC_BLOCK, x, sizeof x);
+
+        uint32_t *words = codes_blk + word_base;
+        memset(words, 0, (size_t)16 * b * sizeof(uint32_t));
+        for (int bk = 0; bk < AGC_BLOCK / B; ++bk) {
+            const float *xb = x + bk * B;
+            float sumsq = bucket_sumsq(xb, B);
+            /* a bucket whose sum of squares is below the smallest normal
+             * number, or not finite, is sent as all-zero with scale 0 */
+            int finite = (sumsq == sumsq) && (sumsq != INFINITY);
+            int flushed = !(finite && sumsq >= 1.17549435e-38f);
+            if (!finite) status |= AGC_ORACLE_STATUS_NONFINITE;
+            float S = flushed ? 0.0f : sqrtf(sumsq);
+            scales_blk[i * (AGC_BLOCK / B) + bk] = S;
+            float inv = flushed ? 0.0f : agc_oracle_inv_scale(S, b);
+            for (int t = 0; t < B; ++t) {
+                int o = bk * B + t;
+                int pos = stream_pos_in_block(o);
+                uint32_t code;
+                if (flushed) {
+                    code = zero_code(b);
+                } else {
+                    uint32_t u = agc_oracle_uniform15(seed, round, (uint32_t)i,
+                                                      (uint64_t)q * AGC_BLOCK + (uint64_t)pos);
+                    code = agc_oracle_quantize_one(xb[t], inv, b, u);
+                    if (code > 2u * zero_code(b) + (b == 1 ? 1u : 0u)) status |= AGC_ORACLE_STATUS_RANGE;
+                    code &= (1u << b) - 1u;
+                }
+                int bit = pos * b;
+                words[bit >> 5] |= code << (bit & 31);
+                if ((bit & 31) + b > 32) words[(bit >> 5) + 1] |= code >> (32 - (bit & 31));
+            }
+        }
+        word_base += 16 * b;
+    }
+    return status;
+}
+
+/* read the code at stream position pos (0..511) of a block of one worker */
+static inline uint32_t read_code(const uint32_t *words, int pos, int b)
+{
+    int bit = pos * b;
+    uint64_t w = words[bit >> 5];
+    if ((bit & 31) + b > 32) w |= (uint64_t)words[(bit >> 5) + 1] << 32;
+    return (uint32_t)(w >> (bit & 31)) & ((1u << b) - 1u);
+}
+
+/*
+ * Unpack + dequantise + masked decode of ONE pack block for one straggler
+ * realisation: ghat[o] = sum over received workers i (ascending) of
+ * w_i * S_{i,bucket(o)} * (level / L_i)   (Sec. II-A decode with Eq. quant_def).
+ *   mask   n bytes, 1 = received (non-straggler), 0 = straggler
+ */
+void agc_oracle_decode_block(int n, const uint8_t *bits, int B, const float *w,
+                             const uint8_t *mask, const uint32_t *codes_blk,
+                             const float *scales_blk, float *ghat_blk)
+{
+    for (int o = 0; o < AGC_BLOCK; ++o) {
+        int pos = stream_pos_in_block(o);
+        int bk = o / B;
+        float acc = 0.0f;
+        int word_base = 0;
+        for (int i = 0; i < n; ++i) {
+            int b = bits[i];
+            if (mask[i]) {
+                float S = scales_blk[i * (AGC_BLOCK / B) + bk];
+                float cstep = (w[i] * S) * dec_step(b);
+                float level = (float)read_code(codes_blk + word_base, pos, b) - dec_offset(b);
+                acc = fmaf(cstep, level, acc);
+            }
+            word_base += 16 * b;
+        }
+        ghat_blk[o] = acc;
+    }
+}
+
+/* ---- whole-vector drivers (loop over pack blocks, gather/scatter) ---- */
+
+int64_t agc_oracle_num_blocks(int64_t d) { return (d + AGC_BLOCK - 1) / AGC_BLOCK; }
+
+/* words in worker i's message and its word offset inside the concatenation */
+int64_t agc_oracle_worker_words(int64_t d, int b) { return agc_oracle_num_blocks(d) * 16 * b; }
+
+/*
+ * Full encode: G is k x d with row stride ld. codes: concatenated messages
+ * (worker i at word offset sum_{i'<i} nblk*16*b_i'); scales: n x nb,
+ * nb = ceil(d/B). x_out optional n x d. Returns status bits.
+ */
+uint32_t agc_oracle_encode_quantize(int n, int k, int64_t d, const int32_t *row_ptr,
+                                    const int32_t *col_idx, const float *a, const uint8_t *bits,
+                                    int B, uint64_t seed, uint64_t round, const float *G,
+                                    int64_t ld, uint32_t *codes, float *scales, float *x_out)
+{
+    const int64_t nblk = agc_oracle_num_blocks(d);
+    const int64_t nb = (d + B - 1) / B;
+    const int bpb = AGC_BLOCK / B;
+    int sumb = 0;
+    for (int i = 0; i < n; ++i) sumb += bits[i];
+    float *Gblk = (float *)malloc((size_t)k * AGC_BLOCK * sizeof(float));
+    uint32_t *cblk = (uint32_t *)malloc((size_t)16 * sumb * sizeof(uint32_t));
+    float *sblk = (float *)malloc((size_t)n * bpb * sizeof(float));
+    float *xblk = x_out ? (float *)malloc((size_t)n * AGC_BLOCK * sizeof(float)) : NULL;
+    uint32_t status = 0;
+    for (int64_t q = 0; q < nblk; ++q) {
+        for (int j = 0; j < k; ++j)
+            for (int o = 0; o < AGC_BLOCK; ++o) {
+                int64_t m = q * AGC_BLOCK + o;
+                Gblk[(int64_t)j * AGC_BLOCK + o] = m < d ? G[(int64_t)j * ld + m] : 0.0f;
+            }
+        status |= agc_oracle_encode_block(n, row_ptr, col_idx, a, bits, B, seed, round, q, Gblk,
+                                          cblk, sblk, xblk);
+        int64_t woff = 0;
+        int wb = 0;
+        for (int i = 0; i < n; ++i) {
+            memcpy(codes + woff + q * 16 * bits[i], cblk + wb, (size_t)16 * bits[i] * sizeof(uint32_t));
+            for (int bk = 0; bk < bpb; ++bk)
+                if (q * bpb + bk < nb) scales[(int64_t)i * nb + q * bpb + bk] = sblk[i * bpb + bk];
+            if (x_out)
+                for (int o = 0; o < AGC_BLOCK; ++o)
+                    if (q * AGC_BLOCK + o < d)
+                        x_out[(int64_t)i * d + q * AGC_BLOCK + o] = xblk[(int64_t)i * AGC_BLOCK + o];
+            woff += nblk * 16 * bits[i];
+            wb += 16 * bits[i];
+        }
+    }
+    free(Gblk); free(cblk); free(sblk); free(xblk);
+    return status;
+}
+
+/*
+ * Full decode for R straggler realisations against one set of messages.
+ *   masks R x n; ghat (optional) R x d; beta (optional) d, updated in place by
+ *   beta <- beta - lr[r]*ghat_r for r = 0..R-1 in order (Eq. update_param, the
+ *   gradient being the SUM over partitions).
+ */
+void agc_oracle_decode(int n, int64_t d, const uint8_t *bits, int B, const float *w,
+                       const uint8_t *masks, int R, const float *lr, const uint32_t *codes,
+                       const float *scales, float *ghat, float *beta)
+{
+    const int64_t nblk = agc_oracle_num_blocks(d);
+    const int64_t nb = (d + B - 1) / B;
+    const int bpb = AGC_BLOCK / B;
+    int sumb = 0;
+    for (int i = 0; i < n; ++i) sumb += bits[i];
+    uint32_t *cblk = (uint32_t *)malloc((size_t)16 * sumb * sizeof(uint32_t));
+    float *sblk = (float *)malloc((size_t)n * bpb * sizeof(float));
+    float gblk[AGC_BLOCK];
+    for (int64_t q = 0; q < nblk; ++q) {
+        int64_t woff = 0;
+        int wb = 0;
+        for (int i = 0; i < n; ++i) {
+            memcpy(cblk + wb, codes + woff + q * 16 * bits[i], (size_t)16 * bits[i] * sizeof(uint32_t));
+            for (int bk = 0; bk < bpb; ++bk)
+                sblk[i * bpb + bk] = (q * bpb + bk < nb) ? scales[(int64_t)i * nb + q * bpb + bk] : 0.0f;
+            woff += nblk * 16 * bits[i];
+            wb += 16 * bits[i];
+        }
+        for (int r = 0; r < R; ++r) {
+            agc_oracle_decode_block(n, bits, B, w, masks + (int64_t)r * n, cblk, sblk, gblk);
+            for (int o = 0; o < AGC_BLOCK; ++o) {
+                int64_t m = q * AGC_BLOCK + o;
+                if (m >= d) break;
+                if (ghat) ghat[(int64_t)r * d + m] = gblk[o];
+                if (beta) beta[m] = fmaf(-lr[r], gblk[o], beta[m]);
+            }
+        }
+    }
+    free(cblk); free(sblk);
+}
+
+/* dequantise one worker's whole message into q_i (length d); used by the
+ * quantiser pins (unbiasedness, variance) */
+void agc_oracle_dequantize_worker(int64_t d, int b, int B, const uint32_t *codes_i,
+                                  const float *scales_i, float *out)
+{
+    for (int64_t m = 0; m < d; ++m) {
+        int64_t q = m / AGC_BLOCK;
+        int pos = stream_pos_in_block((int)(m % AGC_BLOCK));
+        float level = (float)read_code(codes_i + q * 16 * b, pos, b) - dec_offset(b);
+        out[m] = (scales_i[m / B] * dec_step(b)) * level;
+    }
+}

@@ -1,0 +1,256 @@
+"""Pins of the design-time oracle (float64): Theorem 1, the interval
+construction, unbiasedness by exact enumeration of straggler patterns, the
+bounds of Lemma 1 / Lemma 2 by Monte-Carlo, the DP allocator by brute force,
+Algorithm 1 by its properties, the two-track decoder by its optimality."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import design as od
+from oracle import roundpath as orp
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_interval_construction_worked_example():
+    rows = []
+    with open(os.path.join(GOLDEN, "interval_example.txt")) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            if line.startswith("Y"):
+                Y = [float(t) for t in line.split()[1:]]
+            else:
+                rows.append([float(t) for t in line.split()])
+    alpha = od.interval_alpha(Y, 3)
+    assert np.allclose(alpha, np.array(rows), atol=1e-15)
+
+
+@pytest.mark.parametrize("n,k", [(4, 4), (6, 10), (10, 10), (16, 16), (50, 50), (7, 3)])
+def test_theorem1_structure_and_sparsity(n, k):
+    """Row sums Y_i > 0 with sum k, column sums 1, alpha >= 0, at most n+k-1
+    non-zeros (Sec. III-A), objective = k^2 / sum c^-1 (Lemma 2)."""
+    rng = np.random.default_rng(n * 100 + k)
+    p = rng.uniform(0.02, 0.6, n)
+    bits = rng.integers(2, 9, n)
+    Y = od.optimal_row_sums(p, bits, k, 512)
+    assert (Y > 0).all() and abs(Y.sum() - k) < 1e-12
+    alpha = od.interval_alpha(Y, k)
+    assert (alpha >= 0).all()
+    assert np.abs(alpha.sum(1) - Y).max() < 1e-12
+    assert np.abs(alpha.sum(0) - 1).max() < 1e-12
+    assert np.count_nonzero(alpha > 1e-12) <= n + k - 1
+    c = od.c_coeff(p, bits, 512)
+    assert abs(od.structure_objective(alpha, c) - od.optimal_objective(c, k)) < 1e-9 * od.optimal_objective(c, k)
+    # any other feasible alpha is no better (convexity): random feasible perturbations
+    for _ in range(20):
+        other = rng.random((n, k))
+        other /= other.sum(0, keepdims=True)
+        assert od.structure_objective(other, c) >= od.structure_objective(alpha, c) * (1 - 1e-12)
+    A, w = od.physical_coefficients(alpha, p)
+    assert od.unbiasedness_residual(A, w, p) < 1e-12
+
+
+def test_homogeneous_special_case():
+    """p_i = p, b_i = b, n = k: Y_i = 1, the interval code is the identity
+    assignment; on a cyclic-s support the optimum spreads each partition
+    evenly, alpha = 1/s."""
+    n = 8
+    p = np.full(n, 0.2)
+    bits = np.full(n, 4)
+    Y = od.optimal_row_sums(p, bits, n, 512)
+    assert np.allclose(Y, 1.0)
+    assert np.allclose(od.interval_alpha(Y, n), np.eye(n))
+    sup = od.cyclic_support(n, n, 3)
+    alpha, _ = od.support_restricted_alpha_reference(od.c_coeff(p, bits, 512), sup, n)
+    dense = np.zeros((n, n))
+    for i, cols in enumerate(sup):
+        dense[i, cols] = 1 / 3
+    assert np.abs(alpha.sum(1) - 1).max() < 1e-6
+    col_err, excess, neg = od.support_kkt_gap(dense, od.c_coeff(p, bits, 512), sup)
+    assert col_err < 1e-12 and excess < 1e-12 and neg >= 0
+
+
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 6])
+def test_unbiasedness_by_exact_enumeration_of_straggler_patterns(n):
+    """E_S[g_hat] = sum_j g_j for ANY gradients when Eq. exp_g2_quant holds:
+    enumerate all 2^n straggler patterns with their probabilities, the quantiser
+    replaced by its expectation (the identity, Sec. II-B)."""
+    rng = np.random.default_rng(n)
+    k = n + 1
+    p = rng.uniform(0.05, 0.5, n)
+    bits = rng.integers(2, 9, n)
+    alpha = od.interval_alpha(od.optimal_row_sums(p, bits, k, 256), k)
+    A, w = od.physical_coefficients(alpha, p)
+    g = rng.standard_normal((k, 7))
+    f = A @ g
+    mean = np.zeros(7)
+    total = 0.0
+    for pat in itertools.product([0, 1], repeat=n):
+        pat = np.array(pat)
+        pr = np.prod(np.where(pat == 1, 1 - p, p))
+        total += pr
+        mean += pr * ((pat * w) @ f)
+    assert abs(total - 1) < 1e-12
+    assert np.abs(mean - g.sum(0)).max() < 1e-6
+    # a wrong decode vector is caught
+    mean_bad = sum(np.prod(np.where(np.array(pat) == 1, 1 - p, p)) * ((np.array(pat) * w * (1 - p)) @ f)
+                   for pat in itertools.product([0, 1], repeat=n))
+    assert np.abs(mean_bad - g.sum(0)).max() > 1e-3
+
+
+def test_support_restricted_reference_on_cyclic_supports():
+    """(c-SP2) on a cyclic support: the general-purpose solver's answer satisfies
+    the KKT certificate, never beats the unrestricted optimum of Theorem 1 and
+    meets it when the support can carry the optimal row sums."""
+    rng = np.random.default_rng(0)
+    n = k = 8
+    p = rng.uniform(0.05, 0.5, n)
+    bits = rng.integers(2, 9, n)
+    c = od.c_coeff(p, bits, 512)
+    sup = od.cyclic_support(n, k, 3)
+    alpha, val = od.support_restricted_alpha_reference(c, sup, k)
+    col_err, excess, neg = od.support_kkt_gap(alpha, c, sup)
+    assert col_err < 1e-8 and excess < 1e-4 and neg >= 0
+    assert val >= od.optimal_objective(c, k) * (1 - 1e-9)
+    # near-homogeneous workers: row sums near 1 fit into s = 3 columns
+    p2 = np.full(n, 0.2) + rng.uniform(-0.01, 0.01, n)
+    c2 = od.c_coeff(p2, np.full(n, 4), 512)
+    _, val2 = od.support_restricted_alpha_reference(c2, sup, k)
+    assert abs(val2 - od.optimal_objective(c2, k)) < 1e-6 * val2
+
+
+def test_lemma1_and_lemma2_bounds_hold_monte_carlo():
+    """E||g - g_hat||^2 <= Lemma 1 bound = Lemma 2 bound at the optimal structure,
+    with ||g_j||^2 <= C, over random straggler patterns and quantiser rounds,
+    through the real encode / quantise / decode path (phi uses the bucket size)."""
+    rng = np.random.default_rng(12)
+    n = k = 6
+    d, B = 512, 128
+    p = rng.uniform(0.05, 0.4, n)
+    bits = np.array([2, 3, 4, 4, 6, 8], np.uint8)
+    alpha = od.interval_alpha(od.optimal_row_sums(p, bits, k, B), k)
+    rp, ci, vals = od.alpha_to_csr(alpha)
+    A = od.csr_to_dense(rp, ci, vals, k)
+    _, w = od.physical_coefficients(A, p)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    G /= np.linalg.norm(G, axis=1, keepdims=True).astype(np.float32)  # C = 1
+    g = G.astype(np.float64).sum(0)
+    rounds = 1500
+    err = 0.0
+    mean = np.zeros(d)
+    for t in range(rounds):
+        codes, scales, st, _ = orp.encode_quantize(rp, ci, vals.astype(np.float32), bits, B, 5, t, G)
+        mask = (rng.random(n) >= p).astype(np.uint8)
+        gh, _ = orp.decode(d, bits, B, w.astype(np.float32), mask[None], codes, scales)
+        err += np.sum((gh[0] - g) ** 2)
+        mean += gh[0]
+    err /= rounds
+    b1 = od.lemma1_bound(A, w, p, bits, B, C=1.0)
+    b2 = od.lemma2_bound(p, bits, k, B, C=1.0)
+    assert abs(b1 - b2) < 1e-6 * b2
+    assert err <= b1
+    assert err > 0.02 * b1  # the bound is not vacuous here
+    assert np.abs(mean / rounds - g).max() < 6 * np.sqrt(b1 / rounds)
+
+
+def test_phi_and_utility_shapes():
+    """phi(z) = l / (4 (2^(z-1)-1)^2); h_i strictly decreasing in p_i (Sec. III-B)
+    and increasing in the bits."""
+    assert od.phi(2, 100) == 25.0
+    assert od.phi(3, 36) == 1.0
+    assert abs(od.phi(8, 4 * 127 * 127) - 1.0) < 1e-15
+    for r in range(6):
+        hs = [od.h_utility(p, r, 512) for p in (0.05, 0.1, 0.2, 0.4)]
+        assert all(x > y for x, y in zip(hs, hs[1:]))
+    assert all(od.h_utility(0.2, r + 1, 512) > od.h_utility(0.2, r, 512) for r in range(6))
+
+
+@pytest.mark.parametrize("n,zres", [(2, 5), (3, 7), (4, 10), (5, 6), (5, 10)])
+def test_dp_allocator_is_exact_by_brute_force(n, zres):
+    rng = np.random.default_rng(n * 31 + zres)
+    for dim in (16, 512, 100000):
+        p = rng.uniform(0.01, 0.6, n)
+        bits, F = od.bit_allocate_dp(p, 2 * n + zres, dim)
+        bits_bf, F_bf = od.bit_allocate_bruteforce(p, 2 * n + zres, dim)
+        assert abs(F - F_bf) <= 1e-12 * abs(F_bf)
+        assert bits.sum() == 2 * n + zres and (bits >= 2).all()
+        assert abs(od.allocation_value(p, bits.astype(int) - 2, dim) - F) <= 1e-12 * abs(F)
+    p = rng.uniform(0.01, 0.6, n)
+    bits, F = od.bit_allocate_dp(p, 2 * n + zres, 512, b_max=2 + (zres + n - 1) // n + 1)
+    bits_bf, F_bf = od.bit_allocate_bruteforce(p, 2 * n + zres, 512, b_max=2 + (zres + n - 1) // n + 1)
+    assert abs(F - F_bf) <= 1e-12 * abs(F_bf) and bits.max() <= 2 + (zres + n - 1) // n + 1
+
+
+@pytest.mark.parametrize("n", [10, 50])
+def test_low_complexity_allocator_properties(n):
+    """Algorithm 1: feasible, at least as good as equal allocation over all
+    workers and as concentrating on the single most reliable worker, and near the
+    DP optimum (the paper: near-optimal, consistently matching DP)."""
+    rng = np.random.default_rng(n)
+    worst = 1.0
+    for trial in range(4 if n == 10 else 2):
+        psi = rng.uniform(0.1, 2.0, n)
+        p = np.exp(-psi * 0.1)  # shifted-exponential model, tau_th = 1.1 (Sec. VI)
+        p = np.minimum(p, 0.95)
+        for zres in (n, 3 * n):
+            for dim in ((128, 4096) if n == 10 else (512,)):
+                bits, F = od.bit_allocate_low_complexity(p, 2 * n + zres, dim)
+                assert bits.sum() == 2 * n + zres and (bits >= 2).all()
+                base, rem = divmod(zres, n)
+                order = np.argsort(p, kind="stable")
+                r_eq = np.zeros(n, int)
+                r_eq[order] = base + (np.arange(n) < rem)
+                assert F >= od.allocation_value(p, r_eq, dim) * (1 - 1e-12)
+                r_one = np.zeros(n, int)
+                r_one[order[0]] = zres
+                assert F >= od.allocation_value(p, r_one, dim) * (1 - 1e-12)
+                _, F_dp = od.bit_allocate_dp(p, 2 * n + zres, dim)
+                assert F <= F_dp * (1 + 1e-12)
+                worst = min(worst, F / F_dp)
+    assert worst >= 0.99
+
+
+def test_low_complexity_allocator_respects_cap():
+    rng = np.random.default_rng(3)
+    p = rng.uniform(0.02, 0.5, 16)
+    bits, F = od.bit_allocate_low_complexity(p, 64, 512, b_max=8)
+    assert bits.sum() == 64 and bits.min() >= 2 and bits.max() <= 8
+    _, F_dp = od.bit_allocate_dp(p, 64, 512, b_max=8)
+    assert F_dp * 0.99 <= F <= F_dp * (1 + 1e-12)
+
+
+def test_eta_balance_formula():
+    """eta = mean(p) * 4 (2^(Z_tot/n - 1) - 1)^2 / l makes eta*phi(Z_tot/n) = mean(p)."""
+    p = np.array([0.1, 0.3, 0.2, 0.4])
+    eta = od.eta_balance(p, 16, 1000)
+    assert abs(eta * od.phi(4, 1000) - p.mean()) < 1e-15
+    c = od.c_coeff(p, [4] * 4, 1000, eta)
+    assert np.allclose(c, (p + p.mean()) / (1 - p))
+
+
+def test_two_track_decoder_is_the_minimiser():
+    """v* minimises Lambda*Bias + Var over R^n (zero gradient, no better point
+    nearby) and satisfies Var(v*) <= Var(w), Bias(v*) <= Var(w)/Lambda (Prop. 2)."""
+    rng = np.random.default_rng(9)
+    n = k = 7
+    p = rng.uniform(0.05, 0.5, n)
+    bits = rng.integers(2, 8, n)
+    alpha = od.interval_alpha(od.optimal_row_sums(p, bits, k, 256), k)
+    A, w = od.physical_coefficients(alpha, p)
+    for lam in (0.1, 1.0, 10.0):
+        v = od.two_track_decoder(A, p, bits, 256, lam)
+        M, bias, var = od.two_track_objective(v, A, p, bits, 256, lam)
+        Mw, bw, vw = od.two_track_objective(w, A, p, bits, 256, lam)
+        assert bw < 1e-20 and var <= vw and bias <= vw / lam and M <= Mw
+        for _ in range(50):
+            v2 = v + 1e-3 * rng.standard_normal(n)
+            assert od.two_track_objective(v2, A, p, bits, 256, lam)[0] >= M
+        eps = 1e-6
+        grad = [(od.two_track_objective(v + eps * np.eye(n)[i], A, p, bits, 256, lam)[0]
+                 - od.two_track_objective(v - eps * np.eye(n)[i], A, p, bits, 256, lam)[0]) / (2 * eps)
+                for i in range(n)]
+        assert np.abs(grad).max() < 1e-6 * max(M, 1.0)

@@ -1,0 +1,416 @@
+"""Pins of the per-round CPU oracle against facts the paper and the mathematics
+fix (no GPU). A plausible mistake in the oracle - wrong Philox constant, wrong
+sign or offset in the fixed-point rounding, swapped index in packing or in the
+decode sum - fails at least one of these."""
+import ctypes
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import roundpath as orp
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def identity_code(n):
+    return np.arange(n + 1, dtype=np.int32), np.arange(n, dtype=np.int32), np.ones(n, np.float32)
+
+
+# ------------------------------------------------------------------ Philox
+def _curand_host():
+    for name in ("libcurand.so.10", "/usr/local/cuda/lib64/libcurand.so.10", "libcurand.so"):
+        try:
+            return ctypes.CDLL(name)
+        except OSError:
+            continue
+    return None
+
+
+def test_philox_matches_curand_host_generator():
+    """Independent library routine: cuRAND's HOST Philox4_32_10 generator (runs on
+    the CPU). Found by observation: its block t (4 words) is the Philox block of
+    counter (t // 65536, 0, t % 65536, 0) under key = (seed_lo, seed_hi)."""
+    lib = _curand_host()
+    if lib is None:
+        pytest.skip("libcurand not found")
+    for seed in (0, 1, 0x123456789ABCDEF0, 0xDEADBEEFCAFEF00D):
+        gen = ctypes.c_void_p()
+        assert lib.curandCreateGeneratorHost(ctypes.byref(gen), 161) == 0
+        assert lib.curandSetPseudoRandomGeneratorSeed(gen, ctypes.c_ulonglong(seed)) == 0
+        nblk = 3 * 65536 + 17
+        out = np.zeros(4 * nblk, np.uint32)
+        assert lib.curandGenerate(gen, out.ctypes.data_as(ctypes.c_void_p),
+                                  ctypes.c_size_t(out.size)) == 0
+        lib.curandDestroyGenerator(gen)
+        out = out.reshape(-1, 4)
+        key = [seed & 0xFFFFFFFF, seed >> 32]
+        rng = np.random.default_rng(seed & 0xFFFF)
+        picks = np.unique(np.concatenate([[0, 1, 65535, 65536, 65537, nblk - 1],
+                                          rng.integers(0, nblk, 3000)]))
+        for t in picks:
+            t = int(t)
+            got = orp.philox4x32_10([t // 65536, 0, t % 65536, 0], key)
+            assert (got == out[t]).all(), (seed, t)
+
+
+def test_philox_is_a_bijection_and_diffuses():
+    """For a fixed key Philox is a permutation of the counter space: distinct
+    counters give distinct blocks; flipping one counter bit flips about half of
+    the 128 output bits."""
+    key = [0xA4093822, 0x299F31D0]
+    seen = set()
+    rng = np.random.default_rng(0)
+    flips = []
+    for _ in range(2000):
+        ctr = rng.integers(0, 2 ** 32, 4, dtype=np.uint64).astype(np.uint32)
+        a = orp.philox4x32_10(ctr, key)
+        seen.add(a.tobytes())
+        c2 = ctr.copy()
+        word, bit = rng.integers(0, 4), rng.integers(0, 32)
+        c2[word] ^= np.uint32(1 << bit)
+        b = orp.philox4x32_10(c2, key)
+        flips.append(sum(bin(int(x) ^ int(y)).count("1") for x, y in zip(a, b)))
+    assert len(seen) == 2000
+    assert 60 < np.mean(flips) < 68
+
+
+def test_uniform15_lane_selection_and_uniformity():
+    """Eight stream positions share one block; even positions take the low 15 bits
+    of their word, odd ones the high 15 bits. Each draw is in [0, 2^15) and the
+    draws are uniform (chi-square on 64 bins)."""
+    seed, rnd, worker = 0x0123456789ABCDEF, (7 << 32) | 5, 3
+    for pos in (0, 1, 2, 7, 8, 1234567, (1 << 33) + 5):
+        blk = orp.philox4x32_10([(pos >> 3) & 0xFFFFFFFF, worker, rnd & 0xFFFFFFFF, rnd >> 32],
+                                [seed & 0xFFFFFFFF, seed >> 32])
+        word = int(blk[(pos & 7) >> 1])
+        want = (word >> 17) if pos & 1 else (word & 0x7FFF)
+        assert orp.uniform15(seed, rnd, worker, pos) == want
+    u = np.array([orp.uniform15(11, 0, 0, pos) for pos in range(200_000)])
+    assert u.min() >= 0 and u.max() < 32768
+    hist = np.bincount(u >> 9, minlength=64)
+    chi2 = ((hist - len(u) / 64) ** 2 / (len(u) / 64)).sum()
+    assert chi2 < 120  # 63 dof: mean 63, 120 is beyond the 99.99th percentile
+    # different workers / rounds / seeds give different streams
+    assert orp.uniform15(11, 0, 1, 0) != orp.uniform15(11, 0, 0, 0) or \
+        orp.uniform15(11, 0, 1, 8) != orp.uniform15(11, 0, 0, 8)
+    assert [orp.uniform15(11, 1, 0, t) for t in range(8)] != [orp.uniform15(11, 0, 0, t) for t in range(8)]
+    assert [orp.uniform15(12, 0, 0, t) for t in range(8)] != [orp.uniform15(11, 0, 0, t) for t in range(8)]
+
+
+# ------------------------------------------------------------------ quantiser, one coordinate
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_quantizer_exactly_unbiased_by_enumeration_of_all_uniforms(b):
+    """E[Q(x) | x] = x (Sec. II-B). Brute force: enumerate ALL 2^15 values of the
+    uniform for one coordinate; the mean dequantised value equals x up to the
+    2^-15-of-a-step resolution of the uniform, and the variance equals the
+    closed form step^2 * f(1-f) <= step^2/4 (the paper's per-coordinate bound)."""
+    rng = np.random.default_rng(b)
+    S = np.float32(3.7)
+    inv = np.float32(orp.inv_scale(S, b))
+    step = (S / ((1 << (b - 1)) - 1)) if b >= 2 else 2.0 * S
+    xs = np.concatenate([rng.uniform(-S, S, 6), [0.0, S, -S, S / 3, -S * 0.999]]).astype(np.float32)
+    for x in xs:
+        vals = np.array([orp.dequantize_one(orp.quantize_one(float(x), float(inv), b, u), float(S), b)
+                         for u in range(0, 32768)], np.float64)
+        assert abs(vals.mean() - float(x)) <= step * (2.0 ** -15) + 2e-6 * float(S), (b, x)
+        y = (float(x) / float(S)) * (((1 << (b - 1)) - 1) if b >= 2 else 0.5)
+        if b == 1:
+            y += 0.5
+        f = y - np.floor(y)
+        assert abs(vals.var() - step ** 2 * f * (1 - f)) <= step ** 2 * 2e-4
+        assert vals.var() <= step ** 2 / 4 + 1e-12
+        # only the two neighbouring grid points occur
+        assert len(np.unique(vals)) <= 2
+
+
+@pytest.mark.parametrize("b", [2, 3, 5, 8])
+def test_quantizer_matches_plain_float64_definition(b):
+    """Eq. rv_quant written out in float64: level = floor(L*x/S + u/2^15). The
+    oracle's single-fma fixed-point form must give the same level except when
+    L*x/S*2^15 + u lies within rounding distance of a multiple of 2^15."""
+    rng = np.random.default_rng(100 + b)
+    L = (1 << (b - 1)) - 1
+    S = np.float32(0.0123)
+    inv = np.float32(orp.inv_scale(S, b))
+    mism = 0
+    N = 20000
+    for _ in range(N):
+        x = np.float32(rng.uniform(-float(S), float(S)))
+        u = int(rng.integers(0, 32768))
+        code = orp.quantize_one(float(x), float(inv), b, u)
+        t = L * float(x) / float(S) * 32768.0 + u
+        want = int(np.floor(t / 32768.0)) + L
+        if code != want:
+            mism += 1
+            assert abs(code - want) == 1
+            assert abs(t / 32768.0 - round(t / 32768.0)) < 1e-4
+    assert mism <= N * 2e-3
+
+
+def test_quantizer_special_cases():
+    """One-hot vector: the non-zero coordinate is sent as exactly +-S (code 2L or 0);
+    zero vector: scale 0 and every code the zero level; scaling the input by a
+    power of two leaves the codes unchanged and scales the norm."""
+    rp, ci, a = identity_code(1)
+    for b in (2, 4, 8):
+        L = (1 << (b - 1)) - 1
+        G = np.zeros((1, 512), np.float32)
+        G[0, 77] = -2.5
+        codes, scales, st, _ = orp.encode_quantize(rp, ci, a, [b], 512, 5, 0, G)
+        assert st == 0 and scales[0, 0] == np.float32(2.5)
+        deq = orp.dequantize_worker(512, b, 512, codes, scales[0])
+        assert deq[77] == np.float32(-2.5) and np.count_nonzero(deq) == 1
+        G[0, 77] = 2.5
+        codes, scales, st, _ = orp.encode_quantize(rp, ci, a, [b], 512, 5, 0, G)
+        assert orp.dequantize_worker(512, b, 512, codes, scales[0])[77] == np.float32(2.5)
+        Z = np.zeros((1, 512), np.float32)
+        codes, scales, st, _ = orp.encode_quantize(rp, ci, a, [b], 512, 5, 0, Z)
+        assert st == 0 and scales[0, 0] == 0
+        assert (orp.dequantize_worker(512, b, 512, codes, scales[0]) == 0).all()
+        # every b-bit field holds the zero level L
+        bitstr = "".join(format(int(wd), "032b")[::-1] for wd in codes)
+        fields = {int(bitstr[t * b:(t + 1) * b][::-1], 2) for t in range(512)}
+        assert fields == {L}
+    rng = np.random.default_rng(3)
+    G = rng.standard_normal((1, 1024)).astype(np.float32)
+    c1, s1, _, _ = orp.encode_quantize(rp, ci, a, [5], 256, 9, 4, G)
+    c2, s2, _, _ = orp.encode_quantize(rp, ci, a, [5], 256, 9, 4, G * np.float32(2.0 ** -7))
+    assert (c1 == c2).all() and (s2 == s1 * np.float32(2.0 ** -7)).all()
+
+
+def test_nonfinite_and_tiny_buckets_are_flushed():
+    rp, ci, a = identity_code(1)
+    G = np.ones((1, 1024), np.float32)
+    G[0, 600] = np.nan
+    codes, scales, st, _ = orp.encode_quantize(rp, ci, a, [4], 512, 1, 0, G)
+    assert st & orp.STATUS_NONFINITE
+    assert scales[0, 1] == 0 and scales[0, 0] > 0
+    G = np.full((1, 512), 1e-30, np.float32)  # squares underflow
+    codes, scales, st, _ = orp.encode_quantize(rp, ci, a, [4], 512, 1, 0, G)
+    assert st == 0 and scales[0, 0] == 0
+
+
+@pytest.mark.parametrize("B", [128, 256, 512])
+def test_bucket_norm_is_the_l2_norm(B):
+    """Scale = ||x||_2 over the bucket (Eq. quant_def); the last bucket is ragged."""
+    rng = np.random.default_rng(B)
+    d = 3 * 512 + 200
+    G = (rng.standard_normal((1, d)) * 10.0 ** rng.uniform(-3, 3, d)).astype(np.float32)
+    rp, ci, a = identity_code(1)
+    _, scales, st, _ = orp.encode_quantize(rp, ci, a, [4], B, 1, 0, G)
+    nb = (d + B - 1) // B
+    assert scales.shape == (1, nb)
+    for beta in range(nb):
+        ref = np.sqrt(np.sum(G[0, beta * B:(beta + 1) * B].astype(np.float64) ** 2))
+        assert abs(scales[0, beta] - ref) <= 4e-7 * ref
+
+
+def test_codes_never_leave_their_range_on_adversarial_inputs():
+    """|x| <= S must hold for every coordinate so that level stays in [-L, L]:
+    one-hot buckets, equal-magnitude buckets, huge and tiny magnitudes."""
+    rp, ci, a = identity_code(1)
+    rng = np.random.default_rng(5)
+    for b in (1, 2, 8):
+        for trial in range(40):
+            G = np.zeros((1, 512), np.float32)
+            kind = trial % 4
+            mag = np.float32(10.0 ** rng.uniform(-15, 15))
+            if kind == 0:
+                G[0, rng.integers(0, 512)] = mag * rng.choice([-1, 1])
+            elif kind == 1:
+                G[0, :] = mag * rng.choice([-1, 1], 512)
+            elif kind == 2:
+                G[0, :2] = [mag, -mag * np.float32(1e-4)]
+            else:
+                G[0, :] = mag * rng.standard_normal(512)
+            for rnd in range(3):
+                _, _, st, _ = orp.encode_quantize(rp, ci, a, [b], 512, trial, rnd, G)
+                assert st == 0
+
+
+# ------------------------------------------------------------------ vector-level statistics
+def test_unbiasedness_and_variance_bound_monte_carlo():
+    """E[Q(x)] = x and E||Q(x)-x||^2 <= phi(z)||x||^2 with phi = B/(4 L^2) per
+    bucket (Sec. II-B), by Monte-Carlo over rounds; the exact variance
+    sum (S/L)^2 f(1-f) is matched too."""
+    rng = np.random.default_rng(17)
+    d, B, b = 1024, 256, 3
+    L = 3
+    G = rng.standard_normal((1, d)).astype(np.float32)
+    rp, ci, a = identity_code(1)
+    rounds = 3000
+    acc = np.zeros(d)
+    err2 = 0.0
+    for t in range(rounds):
+        codes, scales, _, _ = orp.encode_quantize(rp, ci, a, [b], B, 99, t, G)
+        q = orp.dequantize_worker(d, b, B, codes, scales[0]).astype(np.float64)
+        acc += q
+        err2 += np.sum((q - G[0]) ** 2)
+    mean = acc / rounds
+    S = np.repeat(scales[0].astype(np.float64), B)
+    step = S / L
+    y = np.abs(G[0].astype(np.float64)) / step
+    f = y - np.floor(y)
+    var = step ** 2 * f * (1 - f)
+    z = (mean - G[0]) / np.sqrt(np.maximum(var, 1e-30) / rounds)
+    assert np.abs(z[var > 1e-12]).max() < 5.5
+    assert abs(err2 / rounds - var.sum()) < 0.03 * var.sum()
+    bound = sum(B / (4 * L * L) * np.sum(G[0, t * B:(t + 1) * B].astype(np.float64) ** 2)
+                for t in range(d // B))
+    assert err2 / rounds <= bound
+
+
+# ------------------------------------------------------------------ packing / layout
+def test_stream_position_is_a_block_permutation():
+    pos = [orp.stream_position(m) for m in range(3 * 512)]
+    for q in range(3):
+        assert sorted(pos[q * 512:(q + 1) * 512]) == list(range(q * 512, (q + 1) * 512))
+
+
+def test_hand_built_layout_examples():
+    """Hand-derived from the wire format: offset o = 128c + 4l + e sits at stream
+    position 16l + 4c + e, b bits per position, little-endian words. With b = 8 a
+    one-hot +S coordinate is the byte 0xFE among 0x7F bytes."""
+    rp, ci, a = identity_code(1)
+    cases = {}
+    with open(os.path.join(GOLDEN, "layout_examples.txt")) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if line:
+                m, word, shift = (int(t) for t in line.split())
+                cases[m] = (word, shift)
+    assert len(cases) >= 6
+    for m, (word, shift) in cases.items():
+        G = np.zeros((1, 1024), np.float32)
+        G[0, m] = 1.0
+        codes, _, _, _ = orp.encode_quantize(rp, ci, a, [8], 512, 0, 0, G)
+        expect = np.full(codes.shape, 0x7F7F7F7F, np.uint32)
+        blk = m // 512
+        # the other block holds an all-zero bucket: zero level everywhere as well
+        expect[word] = (0x7F7F7F7F & ~(0xFF << shift)) | (0xFE << shift)
+        assert (codes == expect).all(), m
+        assert word // 128 == blk
+
+
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("d", [1, 511, 512, 513, 1500])
+def test_pack_roundtrip_and_sizes(b, d):
+    """unpack(pack(codes)) reproduces every coordinate to within one quantisation
+    step for every bit width and ragged length; message sizes are whole blocks."""
+    rng = np.random.default_rng(b * 1000 + d)
+    G = rng.standard_normal((1, d)).astype(np.float32)
+    rp, ci, a = identity_code(1)
+    codes, scales, st, x = orp.encode_quantize(rp, ci, a, [b], 128, 3, 1, G, want_x=True)
+    assert st == 0
+    assert (x[0] == G[0]).all()
+    assert codes.size == ((d + 511) // 512) * 16 * b
+    deq = orp.dequantize_worker(d, b, 128, codes, scales[0])
+    S = np.repeat(scales[0], 128)[:d]
+    step = S / ((1 << (b - 1)) - 1) if b >= 2 else 2 * S
+    assert (np.abs(deq - G[0]) <= step * (1 + 1e-6)).all()
+
+
+# ------------------------------------------------------------------ encode / decode
+def test_encode_is_the_weighted_sum_in_partition_order():
+    """f_i = sum_j a_ij g_j (Sec. II-A), checked against float64 and, for the
+    order, against an explicit float32 fma chain on a case where order matters."""
+    rng = np.random.default_rng(2)
+    k, n, d = 5, 3, 700
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-4, 4, (k, 1))).astype(np.float32)
+    rp = np.array([0, 2, 5, 6], np.int32)
+    ci = np.array([0, 3, 1, 2, 4, 4], np.int32)
+    a = rng.uniform(0.1, 2.0, 6).astype(np.float32)
+    _, _, _, x = orp.encode_quantize(rp, ci, a, [4, 4, 4], 128, 1, 0, G, want_x=True)
+    dense = np.zeros((n, k))
+    for i in range(n):
+        for e in range(rp[i], rp[i + 1]):
+            dense[i, ci[e]] = a[e]
+    ref = dense @ G.astype(np.float64)
+    mag = np.abs(dense) @ np.abs(G.astype(np.float64))
+    assert (np.abs(x - ref) <= 3 * 6e-8 * mag + 1e-30).all()
+
+
+def test_decode_special_cases_and_linearity_in_the_mask():
+    """All workers received, identity code, w = 1: g_hat = sum_i Q(g_i). Empty
+    mask: g_hat = 0. Exact enumeration of all 2^n straggler patterns: the
+    probability-weighted mean of the decoded vectors equals
+    sum_i (1-p_i) w_i q_i (the estimator is linear in the indicators)."""
+    rng = np.random.default_rng(4)
+    n, d, B = 4, 1300, 256
+    bits = np.array([2, 3, 4, 8], np.uint8)
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    w = rng.uniform(0.5, 2.0, n).astype(np.float32)
+    G = rng.standard_normal((n, d)).astype(np.float32)
+    rp, ci, a = identity_code(n)
+    codes, scales, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 8, 2, G)
+    off = orp.worker_word_offsets(d, bits)
+    q = np.stack([orp.dequantize_worker(d, int(bits[i]), B, codes[off[i]:off[i + 1]], scales[i])
+                  for i in range(n)]).astype(np.float64)
+    ones = np.ones(n, np.float32)
+    ghat, _ = orp.decode(d, bits, B, ones, np.ones((1, n), np.uint8), codes, scales)
+    assert np.abs(ghat[0] - q.sum(0)).max() <= 1e-5 * np.abs(q).sum(0).max()
+    ghat0, _ = orp.decode(d, bits, B, w, np.zeros((1, n), np.uint8), codes, scales)
+    assert (ghat0 == 0).all()
+    masks = np.array(list(itertools.product([0, 1], repeat=n)), np.uint8)
+    gh, _ = orp.decode(d, bits, B, w, masks, codes, scales)
+    prob = np.prod(np.where(masks == 1, 1 - p, p), axis=1)
+    mean = (prob[:, None] * gh.astype(np.float64)).sum(0)
+    want = (((1 - p) * w.astype(np.float64))[:, None] * q).sum(0)
+    assert np.abs(mean - want).max() <= 2e-6 * np.abs(want).max()
+    # single survivor = that worker's scaled message
+    for i in range(n):
+        m1 = np.zeros((1, n), np.uint8)
+        m1[0, i] = 1
+        g1, _ = orp.decode(d, bits, B, w, m1, codes, scales)
+        assert np.abs(g1[0] - float(w[i]) * q[i]).max() <= 1e-6 * np.abs(q[i]).max() * w[i]
+
+
+def test_batched_decode_equals_single_calls_and_update_rule():
+    """R realisations against one set of messages equal R separate decodes; the
+    fused update is beta <- beta - lr_r * g_hat_r in order (Eq. update_param)."""
+    rng = np.random.default_rng(6)
+    n, d, B = 5, 900, 128
+    bits = np.array([1, 2, 5, 8, 3], np.uint8)
+    w = rng.uniform(0.5, 2.0, n).astype(np.float32)
+    G = rng.standard_normal((n, d)).astype(np.float32)
+    rp, ci, a = identity_code(n)
+    codes, scales, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 1, 0, G)
+    masks = (rng.random((6, n)) > 0.3).astype(np.uint8)
+    lr = rng.uniform(0.01, 0.1, 6).astype(np.float32)
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    gh, beta = orp.decode(d, bits, B, w, masks, codes, scales, lr=lr, beta=beta0)
+    ref = beta0.astype(np.float64).copy()
+    for r in range(6):
+        g1, _ = orp.decode(d, bits, B, w, masks[r:r + 1], codes, scales)
+        assert (g1[0] == gh[r]).all()
+        ref -= float(lr[r]) * gh[r].astype(np.float64)
+    assert np.abs(beta - ref).max() <= 1e-6 * np.abs(ref).max()
+
+
+def test_block_entry_points_agree_with_whole_vector_drivers():
+    rng = np.random.default_rng(8)
+    n, k, d, B = 3, 4, 1100, 256
+    bits = np.array([3, 8, 1], np.uint8)
+    rp = np.array([0, 2, 4, 6], np.int32)
+    ci = np.array([0, 1, 1, 2, 0, 3], np.int32)
+    a = rng.uniform(0.2, 1.0, 6).astype(np.float32)
+    w = rng.uniform(0.5, 2.0, n).astype(np.float32)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    codes, scales, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 21, 3, G)
+    off = orp.worker_word_offsets(d, bits)
+    mask = np.array([1, 0, 1], np.uint8)
+    gh, _ = orp.decode(d, bits, B, w, mask[None], codes, scales)
+    for q in range(3):
+        Gblk = np.zeros((k, 512), np.float32)
+        hi = min(d, (q + 1) * 512)
+        Gblk[:, :hi - q * 512] = G[:, q * 512:hi]
+        cb, sb, _, _ = orp.encode_block(rp, ci, a, bits, B, 21, 3, q, Gblk)
+        wb = 0
+        for i in range(n):
+            nw = 16 * int(bits[i])
+            assert (cb[wb:wb + nw] == codes[off[i] + q * nw: off[i] + (q + 1) * nw]).all()
+            wb += nw
+        gb = orp.decode_block(bits, B, w, mask, cb, sb)
+        assert (gb[:hi - q * 512] == gh[0, q * 512:hi]).all()
