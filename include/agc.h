@@ -1,0 +1,221 @@
+/*
+ * agc.h - C ABI of the B200 coded-gradient library.
+ *
+ * Per-round hot path of joint approximate gradient coding and quantisation for
+ * heterogeneous stragglers: every simulated worker i forms its coded gradient
+ * f_i = sum_j a_ij g_j, quantises it stochastically at b_i bits per coordinate
+ * and bit-packs it; the master unpacks, dequantises and forms the
+ * straggler-masked estimate g_hat = sum_i I_i w_i q_i, optionally fused with
+ * the parameter update. All n workers are simulated on one GPU.
+ *
+ * Letters: n workers, k partitions, d coordinates, b_i bits (the paper writes
+ * k workers, n partitions, l coordinates, z_i bits).
+ *
+ * Conventions for every call
+ *   - returns AGC_OK (0) or a negative AGC_ERR_* code; never aborts, never throws;
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA device
+ *     memory of the current device; the caller owns every buffer it passes, the
+ *     library owns only the plan;
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream);
+ *     device work is enqueued on it and the call returns without synchronising
+ *     unless stated otherwise;
+ *   - a plan may be used from one thread at a time.
+ *
+ * Wire format of the messages (the paper counts bits only; the layout is ours):
+ *   coordinates are grouped in pack blocks of 512; inside a block the coordinate
+ *   at offset o = 128*c + 4*l + e (c < 4, l < 32, e < 4) sits at stream position
+ *   16*l + 4*c + e; worker i's message is a little-endian bit stream over 32-bit
+ *   words with b_i bits per stream position, padded to whole blocks (16*b_i words
+ *   per block); messages are concatenated in worker order; the code of a
+ *   coordinate is level + L_i with level in [-L_i, L_i], L_i = 2^(b_i-1) - 1
+ *   (b_i = 1: the bit of a two-point quantiser {-S, +S}); scales[i*nb + beta] is
+ *   the l2 norm S of bucket beta (bucket = `bucket` consecutive coordinates) of
+ *   worker i's coded gradient, nb = ceil(d / bucket).
+ */
+#ifndef AGC_H
+#define AGC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AGC_OK 0
+#define AGC_ERR_ARG (-1)        /* NULL / out-of-range argument, malformed CSR          */
+#define AGC_ERR_BITS (-2)       /* bits outside 2..8 (1 needs AGC_FLAG_ALLOW_1BIT)      */
+#define AGC_ERR_PROB (-3)       /* a straggler probability outside [0, 1)               */
+#define AGC_ERR_ALIGN (-4)      /* pointer or leading dimension not 16-byte aligned     */
+#define AGC_ERR_UNBIASED (-5)   /* sum_i (1-p_i) w_i a_ij != 1 for some partition j     */
+#define AGC_ERR_CUDA (-6)       /* a CUDA runtime / driver call failed                  */
+#define AGC_ERR_STATE (-7)      /* plan cannot serve this call (e.g. R too large)       */
+#define AGC_ERR_BUDGET (-8)     /* bit budget infeasible for the allocator              */
+#define AGC_ERR_NOMEM (-9)      /* host or device allocation failed                     */
+
+#define AGC_FLAG_ALLOW_1BIT 1u         /* accept b_i = 1 (two-point quantiser; outside the paper)  */
+#define AGC_FLAG_NO_UNBIASED_CHECK 2u  /* skip the check of the unbiasedness condition             */
+#define AGC_FLAG_FORCE_DIRECT 4u       /* always use the direct-load encode kernel (no TMA staging) */
+
+/* bits OR-ed into *status_dev by the kernels */
+#define AGC_STATUS_NONFINITE 1u  /* a bucket had a NaN/Inf sum of squares: sent as zeros, scale 0 */
+#define AGC_STATUS_TIMEOUT 4u    /* a bounded wait inside a kernel expired; outputs are invalid   */
+
+#define AGC_CODE_INTERVAL 0  /* the closed-form sparse construction (support dictated by Y)  */
+#define AGC_CODE_SUPPORT 1   /* the same objective restricted to a caller-given support       */
+
+typedef struct agc_plan agc_plan_t;
+
+/*
+ * agc_plan_create - fix the coding scheme for all rounds.
+ * Paper: Sec. II-A (encoding matrix A = [a_ij], decoding vector w, straggler
+ * probabilities p_i) and Sec. II-B / problem P1 (bits z_i per coordinate).
+ *
+ *   out        receives the plan (host object; owns small device tables)
+ *   n_workers  n >= 1;  k_parts  k >= 1;  d  1 <= d <= 2^31 - 1024 coordinates
+ *   row_ptr    host, n+1 entries: CSR row pointers of A (worker i <-> row i)
+ *   col_idx    host, nnz entries: partition indices, strictly ascending in a row
+ *   a          host, nnz entries: encoding coefficients a_ij (fp32)
+ *   w          host, n entries: decoding coefficients w_i
+ *   p          host, n entries: straggler probabilities, 0 <= p_i < 1
+ *   bits       host, n entries: b_i in 2..8 (1 with AGC_FLAG_ALLOW_1BIT)
+ *   bucket     coordinates per scale: 128, 256 or 512
+ *   seed       key of the counter-based random stream of the stochastic rounding
+ *   flags      AGC_FLAG_*
+ * All host arrays are copied. Unless AGC_FLAG_NO_UNBIASED_CHECK is set the
+ * unbiasedness condition sum_i (1-p_i) w_i a_ij = 1 (Eq. exp_g2_quant) is checked
+ * for every partition in double precision to 1e-5. Synchronous; allocates.
+ */
+int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int64_t d,
+                    const int32_t *row_ptr, const int32_t *col_idx, const float *a,
+                    const float *w, const float *p, const uint8_t *bits, uint32_t bucket,
+                    uint64_t seed, uint32_t flags);
+
+/* Free the plan and its device tables. NULL is allowed. */
+void agc_plan_destroy(agc_plan_t *plan);
+
+/* Bytes of the concatenated messages: sum_i 4 * 16 * b_i * ceil(d/512)
+ * (payload of Sec. II-B: z_i bits per coordinate, padded to whole blocks). */
+size_t agc_codes_bytes(const agc_plan_t *plan);
+/* Bytes of the scales array: 4 * n * ceil(d / bucket) (the norms of Eq. quant_def). */
+size_t agc_scales_bytes(const agc_plan_t *plan);
+/* Byte offset of worker i's message inside the codes buffer (multiple of 64);
+ * i = n gives agc_codes_bytes. Returns (size_t)-1 for a bad index. */
+size_t agc_worker_offset(const agc_plan_t *plan, int i);
+/* 1 if the plan encodes with the TMA-staged kernel, 0 if with the direct-load kernel. */
+int agc_plan_uses_tma(const agc_plan_t *plan);
+
+/*
+ * agc_encode_quantize - one round of all n workers: encode, quantise, pack.
+ * Paper: f_i = sum_{j in B_i} a_ij g_j (Sec. II-A); Q_i of Eq. quant_def with the
+ * stochastic rounding of Eq. rv_quant, per bucket; payload of Sec. II-B.
+ *
+ *   G_dev      device, k rows of d fp32 partial gradients, row j at G_dev + j*ld;
+ *              16-byte aligned; read once
+ *   ld         row stride in elements, >= d and a multiple of 4
+ *   round      iteration counter t; with the plan's seed it fixes every random
+ *              draw (same plan, G and round => same bits)
+ *   codes_dev  device out, agc_codes_bytes bytes, 16-byte aligned
+ *   scales_dev device out, agc_scales_bytes bytes
+ *   status_dev device, one uint32 or NULL: AGC_STATUS_* bits are OR-ed into it
+ * Asynchronous on the stream. Allocates nothing.
+ */
+int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
+                        void *codes_dev, float *scales_dev, uint32_t *status_dev,
+                        void *cuda_stream);
+
+/*
+ * agc_decode - master side: unpack, dequantise, straggler-masked weighted sum,
+ * optional fused parameter update.
+ * Paper: g_hat = sum_i I_i w_i q_i (Sec. II-A), beta <- beta - gamma * g_hat
+ * (Eq. update_param; the gradient is the SUM over partitions).
+ *
+ *   codes_dev, scales_dev  device, as written by agc_encode_quantize; messages
+ *              of stragglers are not read
+ *   masks_dev  device, R x n bytes, 1 = message of worker i arrived in realisation r
+ *   R          number of straggler realisations decoded against the same messages
+ *   lr_host    host, R learning rates gamma_r; required iff beta_dev != NULL
+ *   ghat_dev   device out or NULL: R x d fp32, realisation r at ghat_dev + r*d
+ *   beta_dev   device in/out or NULL: d fp32 parameters, updated by
+ *              beta <- beta - lr[r] * g_hat_r for r = 0..R-1
+ * With R = 1, or whenever ghat_dev is given, sums run over workers in ascending
+ * order with fused multiply-adds (reproducible bit for bit). With R > 1 and only
+ * beta_dev the R updates are applied in one pass through the linear form
+ * beta -= sum_i (sum_r lr_r I_{r,i}) w_i q_i, equal to the sequential updates up
+ * to fp32 rounding. At least one of ghat_dev / beta_dev must be given.
+ * Asynchronous on the stream; R <= 4096.
+ */
+int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+               const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
+               float *beta_dev, void *cuda_stream);
+
+/*
+ * agc_round_host - a whole round through host buffers: copies G to the device,
+ * encodes, decodes one realisation and copies g_hat back. Same operations as
+ * agc_encode_quantize followed by agc_decode (R = 1).
+ *
+ *   G_host     host (pinned memory recommended), k x d fp32, row stride ld_host >= d
+ *   mask_host  host, n bytes
+ *   ghat_host  host out, d fp32
+ *   status_out host out or NULL: AGC_STATUS_* bits of this round
+ * Device staging buffers are allocated inside the plan on first use and reused.
+ * Synchronous: returns after ghat_host is complete.
+ */
+int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_host, uint64_t round,
+                   const uint8_t *mask_host, float *ghat_host, uint32_t *status_out,
+                   void *cuda_stream);
+
+/*
+ * agc_bit_allocate - the low-complexity bit allocation (Algorithm 1): maximise
+ * F = sum_i h_i(r_i), h_i(r) = (1-p_i)/(p_i + phi(r+2)), sum_i b_i = Z_tot,
+ * b_i = r_i + 2 (problem b-SP1), phi(z) = eta * phi_dim / (4 (2^(z-1)-1)^2).
+ *
+ *   n, p       host: workers and their straggler probabilities
+ *   Z_tot      total bits per coordinate over all workers, >= b_min * n
+ *   b_min      minimum bits per worker; the paper's value is 2 (must be 2)
+ *   b_max      cap per worker (<= 8 for this library's packer) or 0 = no cap
+ *   phi_dim    the dimension l in phi: the bucket size when norms are per bucket
+ *   eta        error-balance factor of Sec. V-B (1.0 = the paper's main text)
+ *   bits_out   host out, n entries
+ *   F_out      host out or NULL: the objective value reached
+ * Host only, no CUDA.
+ */
+int agc_bit_allocate(int n, const double *p, int Z_tot, int b_min, int b_max, double phi_dim,
+                     double eta, uint8_t *bits_out, double *F_out);
+
+/* Exact optimum of the same problem by the dynamic programme of Eq. dp_rec,
+ * V[i,r] = max_a V[i-1,r-a] + h_i(a); O(n * Z_res^2). Same arguments. */
+int agc_bit_allocate_dp(int n, const double *p, int Z_tot, int b_min, int b_max, double phi_dim,
+                        double eta, uint8_t *bits_out, double *F_out);
+
+/*
+ * agc_code_build - code weights for given p and bits.
+ * Paper: Theorem 1 (row sums Y_i = c_i^-1 k / sum_m c_m^-1, column sums 1,
+ * c_i = (p_i + eta*phi(b_i)) / (1 - p_i)), the interval-overlap construction of
+ * Sec. III-A, and a_ij = alpha_ij / w~_i, w_i = w~_i / (1 - p_i) with w~_i = 1.
+ *
+ *   mode AGC_CODE_INTERVAL: alpha_i^j = [min{R_i, j} - max{R_{i-1}, j-1}]_+;
+ *        sup_row_ptr / sup_col_idx are ignored (may be NULL).
+ *   mode AGC_CODE_SUPPORT: minimise sum_i c_i (sum_j alpha_ij)^2 subject to
+ *        column sums 1 and alpha >= 0 on the support given as CSR
+ *        (sup_row_ptr n+1 entries, sup_col_idx ascending within a row).
+ *   nnz_cap      capacity of col_out / a_out (n + k - 1 suffices for INTERVAL,
+ *                the support's nnz for SUPPORT)
+ *   row_ptr_out  host out, n+1;  col_out, a_out  host out, up to nnz_cap
+ *   w_out        host out, n;    Y_out  host out or NULL, n: row sums reached
+ * Host only, no CUDA. Entries below 1e-12 are dropped and columns renormalised.
+ */
+int agc_code_build(int n, int k, const double *p, const uint8_t *bits, double phi_dim,
+                   double eta, int mode, const int32_t *sup_row_ptr,
+                   const int32_t *sup_col_idx, int32_t nnz_cap, int32_t *row_ptr_out,
+                   int32_t *col_out, float *a_out, float *w_out, double *Y_out);
+
+/* Human-readable text for an AGC_ERR_* code (static storage). */
+const char *agc_strerror(int code);
+/* Library version: major*10000 + minor*100 + patch. */
+int agc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AGC_H */

@@ -1,0 +1,225 @@
+// Master side: unpack + dequantise + straggler-masked weighted sum over the received
+// workers (Sec. II-A, g_hat = sum_i I_i w_i q_i, with q_i of Eq. quant_def), optionally
+// fused with the parameter update of Eq. update_param.
+//
+// One warp owns one 512-coordinate pack block. Lane l holds the 16 coordinates
+// {128c + 4l + e}, i.e. stream positions 16l..16l+15 of every worker's message, so it
+// reads 16*b_i contiguous bits per worker and never needs another lane's data.
+#include "agc_internal.h"
+
+namespace {
+
+// Add worker's contribution cstep[row] * level to the lane's 16 accumulators.
+template <int BITS>
+__device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int lane,
+                                                  const float (&cstep_row)[4], float (&acc)[16])
+{
+    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS - 1)) - 1u : 0u;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+    constexpr int NACC = (16 * BITS + 31) / 32;
+    uint32_t A[NACC + 1];
+    A[NACC] = 0u;
+    if constexpr (BITS % 2 == 0) {
+        constexpr int NW = BITS / 2;
+        const uint32_t *src = blk_words + lane * NW;
+        if constexpr (NW == 4) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+            A[0] = v.x; A[1] = v.y; A[2] = v.z; A[3] = v.w;
+        } else if constexpr (NW == 2) {
+            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+            A[0] = v.x; A[1] = v.y;
+        } else {
+#pragma unroll
+            for (int t = 0; t < NW; ++t) A[t] = __ldg(src + t);
+        }
+    } else {
+        // a pair of lanes shares BITS words; the odd lane's slice starts at bit 16 of word H
+        constexpr int H = (BITS - 1) / 2;
+        const uint32_t *src = blk_words + (lane >> 1) * BITS + ((lane & 1) ? H : 0);
+        uint32_t W[H + 1];
+#pragma unroll
+        for (int t = 0; t <= H; ++t) W[t] = __ldg(src + t);
+        if (lane & 1) {
+#pragma unroll
+            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
+            A[H] = W[H] >> 16;
+        } else {
+#pragma unroll
+            for (int t = 0; t <= H; ++t) A[t] = W[t];
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+        const int bitpos = t * BITS;
+        const int w = bitpos >> 5, sh = bitpos & 31;
+        uint32_t code;
+        if (sh + BITS <= 32) code = (A[w] >> sh) & MASK;
+        else code = __funnelshift_r(A[w], A[w + 1], sh) & MASK;
+        float level;
+        if constexpr (BITS >= 2)
+            level = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);  // code - L, exact
+        else
+            level = __uint_as_float(0xBF000000u ^ (code << 31));                          // code - 0.5
+        acc[t] = __fmaf_rn(cstep_row[t >> 2], level, acc[t]);
+    }
+}
+
+template <int RB>
+__device__ __forceinline__ void add_worker(const AgcDecParams &P, int worker, float wgt, long long q, int lane,
+                                           float (&acc)[16])
+{
+    const int bits = P.bits[worker];
+    const float dstep = bits >= 2 ? (float)(1.0 / (double)((1 << (bits - 1)) - 1)) : 2.0f;
+    float cstep_row[4];
+#pragma unroll
+    for (int bk = 0; bk < 4 / RB; ++bk) {
+        const long long beta = q * (4 / RB) + bk;
+        const float S = beta < P.nb ? __ldg(P.scales + (long long)worker * P.nb + beta) : 0.0f;
+        const float cs = __fmul_rn(__fmul_rn(wgt, S), dstep);
+#pragma unroll
+        for (int cc = 0; cc < RB; ++cc) cstep_row[bk * RB + cc] = cs;
+    }
+    const uint32_t *blk_words = P.codes + P.word_off[worker] + q * 16 * bits;
+    switch (bits) {
+        case 1: unpack_accumulate<1>(blk_words, lane, cstep_row, acc); break;
+        case 2: unpack_accumulate<2>(blk_words, lane, cstep_row, acc); break;
+        case 3: unpack_accumulate<3>(blk_words, lane, cstep_row, acc); break;
+        case 4: unpack_accumulate<4>(blk_words, lane, cstep_row, acc); break;
+        case 5: unpack_accumulate<5>(blk_words, lane, cstep_row, acc); break;
+        case 6: unpack_accumulate<6>(blk_words, lane, cstep_row, acc); break;
+        case 7: unpack_accumulate<7>(blk_words, lane, cstep_row, acc); break;
+        default: unpack_accumulate<8>(blk_words, lane, cstep_row, acc); break;
+    }
+}
+
+__device__ __forceinline__ void load16(const float *base, long long q, int lane, long long d, bool vec, float (&v)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const long long m = q * AGC_BLOCK + c * 128 + 4 * lane;
+        if (vec && m + 3 < d) {
+            const float4 x = *reinterpret_cast<const float4 *>(base + m);
+            v[4 * c] = x.x; v[4 * c + 1] = x.y; v[4 * c + 2] = x.z; v[4 * c + 3] = x.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[4 * c + e] = (m + e < d) ? base[m + e] : 0.0f;
+        }
+    }
+}
+
+__device__ __forceinline__ void store16(float *base, long long q, int lane, long long d, bool vec, const float (&v)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const long long m = q * AGC_BLOCK + c * 128 + 4 * lane;
+        if (vec && m + 3 < d) {
+            *reinterpret_cast<float4 *>(base + m) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (m + e < d) base[m + e] = v[4 * c + e];
+        }
+    }
+}
+
+// COLLAPSED = false: realisation by realisation, workers in ascending order (the
+// defining order). COLLAPSED = true: one pass with the effective weights
+// weff_i = sum_r lr_r I_{r,i} (R > 1, update only).
+template <int RB, bool COLLAPSED>
+__global__ void __launch_bounds__(256) agc_decode_kernel(const AgcDecParams P)
+{
+    const int lane = threadIdx.x & 31;
+    const long long q = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (q >= P.nblk) return;
+    const bool vec = (P.d & 3) == 0;
+    float acc[16];
+    if (COLLAPSED) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+        for (int i = 0; i < P.n; ++i) {
+            const float we = P.weff[i];
+            if (we != 0.0f) add_worker<RB>(P, i, __fmul_rn(P.w[i], we), q, lane, acc);
+        }
+        float b[16];
+        load16(P.beta, q, lane, P.d, vec, b);
+#pragma unroll
+        for (int t = 0; t < 16; ++t) b[t] = __fsub_rn(b[t], acc[t]);
+        store16(P.beta, q, lane, P.d, vec, b);
+    } else {
+        float b[16];
+        if (P.beta) load16(P.beta, q, lane, P.d, vec, b);
+        for (int r = 0; r < P.R; ++r) {
+#pragma unroll
+            for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+            const uint8_t *mask = P.masks + (long long)r * P.n;
+            for (int i = 0; i < P.n; ++i)
+                if (mask[i]) add_worker<RB>(P, i, P.w[i], q, lane, acc);
+            if (P.ghat) store16(P.ghat + (long long)r * P.d, q, lane, P.d, vec, acc);
+            if (P.beta) {
+                const float lr = P.R == 1 ? P.lr0 : P.lr[r];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) b[t] = __fmaf_rn(-lr, acc[t], b[t]);
+            }
+        }
+        if (P.beta) store16(P.beta, q, lane, P.d, vec, b);
+    }
+}
+
+// weff_i = sum_r lr_r * I_{r,i}, summed in order of r
+__global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *lr, int n, int R, float *weff)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.0f;
+    for (int r = 0; r < R; ++r)
+        if (masks[(long long)r * n + i]) s = __fadd_rn(s, lr[r]);
+    weff[i] = s;
+}
+
+template <bool COLLAPSED>
+void launch(const AgcDecParams &P, int grid, cudaStream_t stream)
+{
+    if (P.rows_per_bucket == 4) agc_decode_kernel<4, COLLAPSED><<<grid, 256, 0, stream>>>(P);
+    else if (P.rows_per_bucket == 2) agc_decode_kernel<2, COLLAPSED><<<grid, 256, 0, stream>>>(P);
+    else agc_decode_kernel<1, COLLAPSED><<<grid, 256, 0, stream>>>(P);
+}
+
+}  // namespace
+
+int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
+                      int R, const float *lr_host, float *ghat, float *beta, cudaStream_t stream)
+{
+    AgcDecParams P;
+    P.bits = plan->d_bits;
+    P.w = plan->d_w;
+    P.word_off = plan->d_word_off;
+    P.codes = static_cast<const uint32_t *>(codes);
+    P.scales = scales;
+    P.masks = masks;
+    P.weff = nullptr;
+    P.ghat = ghat;
+    P.beta = beta;
+    P.d = plan->d;
+    P.nblk = plan->nblk;
+    P.nb = plan->nb;
+    P.n = plan->n;
+    P.R = R;
+    P.rows_per_bucket = plan->bucket / 128;
+    P.lr0 = (beta && lr_host) ? lr_host[0] : 0.0f;
+    P.lr = plan->d_lr;
+    const int grid = (int)((plan->nblk + 7) / 8);
+    const bool collapsed = R > 1 && beta && !ghat;
+    if (beta && R > 1) {
+        if (cudaMemcpyAsync(plan->d_lr, lr_host, sizeof(float) * R, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return AGC_ERR_CUDA;
+    }
+    if (collapsed) {
+        agc_effective_weights_kernel<<<(plan->n + 127) / 128, 128, 0, stream>>>(masks, plan->d_lr, plan->n, R,
+                                                                               plan->d_weff);
+        P.weff = plan->d_weff;
+        launch<true>(P, grid, stream);
+    } else {
+        launch<false>(P, grid, stream);
+    }
+    return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
+}

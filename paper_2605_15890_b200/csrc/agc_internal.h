@@ -1,0 +1,92 @@
+// Private declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <vector>
+
+#include "../../include/agc.h"
+
+#define AGC_BLOCK 512          // coordinates per pack block (one warp task)
+#define AGC_FRAC_BITS 15       // fractional bits of the fixed-point stochastic rounding
+#define AGC_MAX_STAGES 16      // shared-memory ring depth limit of the staged encoder
+#define AGC_MAX_STAGE_ROWS 36  // partition rows per staged tile (36 * 2 KiB = 72 KiB)
+#define AGC_ENC_CONSUMER_WARPS 16
+#define AGC_MAX_R 4096         // straggler realisations per decode call
+
+// Parameters of one encode launch (passed by value; lives in the constant bank).
+struct AgcEncParams {
+    const int32_t *row_ptr;      // n+1
+    const int32_t *col_idx;      // nnz
+    const float *a;              // nnz
+    const uint8_t *bits;         // n
+    const uint8_t *ent_slot;     // nnz: slot of entry's partition row inside its group's tile
+    const long long *word_off;   // n+1: word offset of each worker's message
+    const int32_t *grp_row_ptr;  // n_groups+1
+    const int32_t *grp_rows;     // partition row per tile slot
+    const int32_t *grp_wk_ptr;   // n_groups+1
+    const int32_t *grp_workers;  // workers of each group
+    const float *G;
+    uint32_t *codes;
+    float *scales;
+    uint32_t *status;
+    long long d, ld, nblk, nb;
+    int n, k, n_groups;
+    int rows_per_bucket;         // bucket / 128: 1, 2 or 4
+    int stages, stage_rows;
+    uint32_t round_lo, round_hi;
+    uint32_t rk[20];             // Philox round keys: rk[2r] = key0 + r*W0, rk[2r+1] = key1 + r*W1
+};
+
+struct AgcDecParams {
+    const uint8_t *bits;
+    const float *w;
+    const long long *word_off;
+    const uint32_t *codes;
+    const float *scales;
+    const uint8_t *masks;   // R x n
+    const float *weff;      // n effective weights (collapsed mode) or NULL
+    float *ghat;            // R x d or NULL
+    float *beta;            // d or NULL
+    long long d, nblk, nb;
+    int n, R;
+    int rows_per_bucket;
+    float lr0;              // learning rate of the single realisation (R == 1)
+    const float *lr;        // device, R learning rates (per-realisation mode with beta)
+};
+
+struct agc_plan {
+    int n = 0, k = 0;
+    long long d = 0, nblk = 0, nb = 0;
+    int bucket = 0;
+    uint64_t seed = 0;
+    uint32_t flags = 0;
+    int device = 0, sm_count = 0;
+    std::vector<int32_t> row_ptr, col_idx;
+    std::vector<float> a, w;
+    std::vector<uint8_t> bits;
+    std::vector<long long> word_off;
+    // encode tiling
+    bool use_tma = false;
+    int n_groups = 0, stage_rows = 0, stages = 0;
+    size_t enc_smem = 0;
+    // device tables
+    int32_t *d_row_ptr = nullptr, *d_col_idx = nullptr;
+    float *d_a = nullptr, *d_w = nullptr;
+    uint8_t *d_bits = nullptr, *d_ent_slot = nullptr;
+    long long *d_word_off = nullptr;
+    int32_t *d_grp_row_ptr = nullptr, *d_grp_rows = nullptr, *d_grp_wk_ptr = nullptr, *d_grp_workers = nullptr;
+    // decode scratch
+    float *d_weff = nullptr, *d_lr = nullptr;
+    // staging for the host-buffer entry point (allocated on first use)
+    float *h_G = nullptr, *h_ghat = nullptr, *h_scales = nullptr;
+    void *h_codes = nullptr;
+    uint8_t *h_mask = nullptr;
+    uint32_t *h_status = nullptr;
+    void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled entry point
+};
+
+int agc_launch_encode(agc_plan *plan, const float *G, long long ld, uint64_t round, void *codes,
+                      float *scales, uint32_t *status, cudaStream_t stream);
+int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
+                      int R, const float *lr_host, float *ghat, float *beta, cudaStream_t stream);

@@ -1,0 +1,275 @@
+// Plan object, argument validation, size queries and the host-buffer round.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "agc_internal.h"
+
+int agc_encode_prepare(agc_plan *plan);
+
+namespace {
+
+template <typename T>
+int upload(T **dst, const std::vector<T> &src)
+{
+    const size_t bytes = (src.empty() ? 1 : src.size()) * sizeof(T);
+    if (cudaMalloc(reinterpret_cast<void **>(dst), bytes) != cudaSuccess) return AGC_ERR_NOMEM;
+    if (!src.empty() && cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    return AGC_OK;
+}
+
+// Partition the workers (in order) into groups whose supports together touch at most
+// AGC_MAX_STAGE_ROWS partition rows: one staged tile = (pack block, group). Returns
+// false when some worker's own support is too wide for a tile.
+bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::vector<int32_t> &grp_rows,
+                  std::vector<int32_t> &grp_wk_ptr, std::vector<int32_t> &grp_workers,
+                  std::vector<uint8_t> &ent_slot, int *max_rows)
+{
+    grp_row_ptr.assign(1, 0);
+    grp_wk_ptr.assign(1, 0);
+    grp_rows.clear();
+    grp_workers.clear();
+    ent_slot.assign(pl.col_idx.size(), 0);
+    std::vector<int> slot_of(pl.k, -1);
+    std::vector<int32_t> cur_rows;
+    *max_rows = 0;
+    auto flush = [&]() {
+        if (grp_workers.size() == size_t(grp_wk_ptr.back())) return;
+        for (int32_t r : cur_rows) { grp_rows.push_back(r); slot_of[r] = -1; }
+        grp_row_ptr.push_back(int32_t(grp_rows.size()));
+        grp_wk_ptr.push_back(int32_t(grp_workers.size()));
+        *max_rows = std::max<int>(*max_rows, int(cur_rows.size()));
+        cur_rows.clear();
+    };
+    for (int i = 0; i < pl.n; ++i) {
+        const int e0 = pl.row_ptr[i], e1 = pl.row_ptr[i + 1];
+        if (e1 - e0 > AGC_MAX_STAGE_ROWS) return false;
+        int fresh = 0;
+        for (int e = e0; e < e1; ++e) fresh += slot_of[pl.col_idx[e]] < 0;
+        if (int(cur_rows.size()) + fresh > AGC_MAX_STAGE_ROWS) flush();
+        for (int e = e0; e < e1; ++e) {
+            const int j = pl.col_idx[e];
+            if (slot_of[j] < 0) { slot_of[j] = int(cur_rows.size()); cur_rows.push_back(j); }
+            ent_slot[e] = uint8_t(slot_of[j]);
+        }
+        grp_workers.push_back(i);
+    }
+    flush();
+    return true;
+}
+
+void free_device(agc_plan *p)
+{
+    cudaFree(p->d_row_ptr); cudaFree(p->d_col_idx); cudaFree(p->d_a); cudaFree(p->d_w);
+    cudaFree(p->d_bits); cudaFree(p->d_ent_slot); cudaFree(p->d_word_off);
+    cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_rows); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
+    cudaFree(p->d_weff); cudaFree(p->d_lr);
+    cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
+    cudaFree(p->h_mask); cudaFree(p->h_status);
+}
+
+}  // namespace
+
+extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int64_t d,
+                               const int32_t *row_ptr, const int32_t *col_idx, const float *a,
+                               const float *w, const float *p, const uint8_t *bits, uint32_t bucket,
+                               uint64_t seed, uint32_t flags)
+{
+    if (!out) return AGC_ERR_ARG;
+    *out = nullptr;
+    if (n_workers < 1 || k_parts < 1 || d < 1 || d > (int64_t(1) << 31) - 1024) return AGC_ERR_ARG;
+    if (!row_ptr || !col_idx || !a || !w || !p || !bits) return AGC_ERR_ARG;
+    if (bucket != 128 && bucket != 256 && bucket != 512) return AGC_ERR_ARG;
+    if (row_ptr[0] != 0) return AGC_ERR_ARG;
+    for (int i = 0; i < n_workers; ++i) {
+        if (row_ptr[i + 1] < row_ptr[i]) return AGC_ERR_ARG;
+        for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e) {
+            if (col_idx[e] < 0 || col_idx[e] >= k_parts) return AGC_ERR_ARG;
+            if (e > row_ptr[i] && col_idx[e] <= col_idx[e - 1]) return AGC_ERR_ARG;
+            if (!std::isfinite(a[e])) return AGC_ERR_ARG;
+        }
+        if (!(p[i] >= 0.0f && p[i] < 1.0f)) return AGC_ERR_PROB;
+        if (!std::isfinite(w[i])) return AGC_ERR_ARG;
+        const int lo = (flags & AGC_FLAG_ALLOW_1BIT) ? 1 : 2;
+        if (bits[i] < lo || bits[i] > 8) return AGC_ERR_BITS;
+    }
+    const int nnz = row_ptr[n_workers];
+    if (!(flags & AGC_FLAG_NO_UNBIASED_CHECK)) {
+        // sum_i (1 - p_i) w_i a_ij = 1 for every partition j (Eq. exp_g2_quant)
+        std::vector<double> col(k_parts, 0.0);
+        for (int i = 0; i < n_workers; ++i)
+            for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                col[col_idx[e]] += (1.0 - double(p[i])) * double(w[i]) * double(a[e]);
+        for (int j = 0; j < k_parts; ++j)
+            if (!(std::fabs(col[j] - 1.0) <= 1e-5)) return AGC_ERR_UNBIASED;
+    }
+
+    agc_plan *pl = new (std::nothrow) agc_plan;
+    if (!pl) return AGC_ERR_NOMEM;
+    pl->n = n_workers;
+    pl->k = k_parts;
+    pl->d = d;
+    pl->bucket = int(bucket);
+    pl->seed = seed;
+    pl->flags = flags;
+    pl->nblk = (d + AGC_BLOCK - 1) / AGC_BLOCK;
+    pl->nb = (d + bucket - 1) / bucket;
+    pl->row_ptr.assign(row_ptr, row_ptr + n_workers + 1);
+    pl->col_idx.assign(col_idx, col_idx + nnz);
+    pl->a.assign(a, a + nnz);
+    pl->w.assign(w, w + n_workers);
+    pl->bits.assign(bits, bits + n_workers);
+    pl->word_off.assign(n_workers + 1, 0);
+    for (int i = 0; i < n_workers; ++i) pl->word_off[i + 1] = pl->word_off[i] + pl->nblk * 16 * bits[i];
+
+    int rc = AGC_OK;
+    int smem_optin = 0;
+    if (cudaGetDevice(&pl->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, pl->device) != cudaSuccess) {
+        delete pl;
+        return AGC_ERR_CUDA;
+    }
+
+    std::vector<int32_t> grp_row_ptr, grp_rows, grp_wk_ptr, grp_workers;
+    std::vector<uint8_t> ent_slot;
+    int max_rows = 0;
+    bool stageable = build_groups(*pl, grp_row_ptr, grp_rows, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
+    pl->n_groups = int(grp_row_ptr.size()) - 1;
+    pl->use_tma = false;
+    if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0) {
+        const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16;
+        const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);
+        long long stages = (long long)((size_t(smem_optin) - tail - 1024) / stage_bytes);
+        if (stages > AGC_MAX_STAGES) stages = AGC_MAX_STAGES;
+        cudaDriverEntryPointQueryResult qres;
+        void *fn = nullptr;
+        if (stages >= 2 &&
+            cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && fn) {
+            pl->use_tma = true;
+            pl->stages = int(stages);
+            pl->stage_rows = max_rows;
+            pl->enc_smem = size_t(stages) * stage_bytes + tail;
+            pl->encode_tiled = fn;
+        }
+    }
+
+    if (!rc) rc = upload(&pl->d_row_ptr, pl->row_ptr);
+    if (!rc) rc = upload(&pl->d_col_idx, pl->col_idx);
+    if (!rc) rc = upload(&pl->d_a, pl->a);
+    if (!rc) rc = upload(&pl->d_w, pl->w);
+    if (!rc) rc = upload(&pl->d_bits, pl->bits);
+    if (!rc) rc = upload(&pl->d_ent_slot, ent_slot);
+    if (!rc) rc = upload(&pl->d_word_off, pl->word_off);
+    if (!rc) rc = upload(&pl->d_grp_row_ptr, grp_row_ptr);
+    if (!rc) rc = upload(&pl->d_grp_rows, grp_rows);
+    if (!rc) rc = upload(&pl->d_grp_wk_ptr, grp_wk_ptr);
+    if (!rc) rc = upload(&pl->d_grp_workers, grp_workers);
+    if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
+    if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_lr), sizeof(float) * AGC_MAX_R) != cudaSuccess) rc = AGC_ERR_NOMEM;
+    if (!rc) rc = agc_encode_prepare(pl);
+    if (rc) {
+        free_device(pl);
+        delete pl;
+        return rc;
+    }
+    *out = pl;
+    return AGC_OK;
+}
+
+extern "C" void agc_plan_destroy(agc_plan_t *plan)
+{
+    if (!plan) return;
+    free_device(plan);
+    delete plan;
+}
+
+extern "C" size_t agc_codes_bytes(const agc_plan_t *plan) { return plan ? size_t(plan->word_off[plan->n]) * 4 : 0; }
+extern "C" size_t agc_scales_bytes(const agc_plan_t *plan) { return plan ? size_t(plan->n) * size_t(plan->nb) * 4 : 0; }
+extern "C" size_t agc_worker_offset(const agc_plan_t *plan, int i)
+{
+    if (!plan || i < 0 || i > plan->n) return size_t(-1);
+    return size_t(plan->word_off[i]) * 4;
+}
+extern "C" int agc_plan_uses_tma(const agc_plan_t *plan) { return plan && plan->use_tma ? 1 : 0; }
+
+extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
+                                   void *codes_dev, float *scales_dev, uint32_t *status_dev, void *cuda_stream)
+{
+    if (!plan || !G_dev || !codes_dev || !scales_dev) return AGC_ERR_ARG;
+    if (ld < plan->d) return AGC_ERR_ARG;
+    if ((ld & 3) || (reinterpret_cast<uintptr_t>(G_dev) & 15) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
+        (reinterpret_cast<uintptr_t>(scales_dev) & 3))
+        return AGC_ERR_ALIGN;
+    return agc_launch_encode(plan, G_dev, ld, round, codes_dev, scales_dev, status_dev,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+                          const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
+                          float *beta_dev, void *cuda_stream)
+{
+    if (!plan || !codes_dev || !scales_dev || !masks_dev) return AGC_ERR_ARG;
+    if (R < 1 || (!ghat_dev && !beta_dev) || (beta_dev && !lr_host)) return AGC_ERR_ARG;
+    if (R > AGC_MAX_R) return AGC_ERR_STATE;
+    if ((reinterpret_cast<uintptr_t>(codes_dev) & 15) || (ghat_dev && (reinterpret_cast<uintptr_t>(ghat_dev) & 15)) ||
+        (beta_dev && (reinterpret_cast<uintptr_t>(beta_dev) & 15)))
+        return AGC_ERR_ALIGN;
+    return agc_launch_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host, ghat_dev, beta_dev,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_host, uint64_t round,
+                              const uint8_t *mask_host, float *ghat_host, uint32_t *status_out,
+                              void *cuda_stream)
+{
+    if (!plan || !G_host || !mask_host || !ghat_host || ld_host < plan->d) return AGC_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const long long ld_dev = (plan->d + 3) & ~3LL;
+    if (!plan->h_G) {
+        bool ok = cudaMalloc(reinterpret_cast<void **>(&plan->h_G), sizeof(float) * ld_dev * plan->k) == cudaSuccess &&
+                  cudaMalloc(&plan->h_codes, agc_codes_bytes(plan)) == cudaSuccess &&
+                  cudaMalloc(reinterpret_cast<void **>(&plan->h_scales), agc_scales_bytes(plan)) == cudaSuccess &&
+                  cudaMalloc(reinterpret_cast<void **>(&plan->h_ghat), sizeof(float) * plan->d) == cudaSuccess &&
+                  cudaMalloc(reinterpret_cast<void **>(&plan->h_mask), plan->n) == cudaSuccess &&
+                  cudaMalloc(reinterpret_cast<void **>(&plan->h_status), sizeof(uint32_t)) == cudaSuccess;
+        if (!ok) return AGC_ERR_NOMEM;
+    }
+    if (cudaMemcpy2DAsync(plan->h_G, sizeof(float) * ld_dev, G_host, sizeof(float) * ld_host,
+                          sizeof(float) * plan->d, plan->k, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(plan->h_mask, mask_host, plan->n, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemsetAsync(plan->h_status, 0, sizeof(uint32_t), st) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    int rc = agc_launch_encode(plan, plan->h_G, ld_dev, round, plan->h_codes, plan->h_scales, plan->h_status, st);
+    if (rc) return rc;
+    rc = agc_launch_decode(plan, plan->h_codes, plan->h_scales, plan->h_mask, 1, nullptr, plan->h_ghat, nullptr, st);
+    if (rc) return rc;
+    uint32_t status = 0;
+    if (cudaMemcpyAsync(ghat_host, plan->h_ghat, sizeof(float) * plan->d, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(&status, plan->h_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    if (status_out) *status_out = status;
+    return AGC_OK;
+}
+
+extern "C" const char *agc_strerror(int code)
+{
+    switch (code) {
+        case AGC_OK: return "ok";
+        case AGC_ERR_ARG: return "invalid argument";
+        case AGC_ERR_BITS: return "bits per coordinate out of range";
+        case AGC_ERR_PROB: return "straggler probability outside [0, 1)";
+        case AGC_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+        case AGC_ERR_UNBIASED: return "code violates the unbiasedness condition";
+        case AGC_ERR_CUDA: return "CUDA call failed";
+        case AGC_ERR_STATE: return "plan cannot serve this call";
+        case AGC_ERR_BUDGET: return "bit budget infeasible";
+        case AGC_ERR_NOMEM: return "out of memory";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int agc_version(void) { return 100; }

@@ -1,0 +1,231 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs. Packed codes, scales and the single-realisation decode must be
+bit-exact; the collapsed multi-realisation update must agree to 1e-5 relative."""
+import numpy as np
+import pytest
+
+from oracle import design as od
+from oracle import roundpath as orp
+from synth import configs as cfgs
+from tests import _codes
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def agc():
+    import paper_2605_15890_b200 as m
+    return m
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+    return t
+
+
+def run_both(agc, torch, G_host, code, p, bits, B, seed, rnd, masks, flags=0, d=None, lr=None, beta0=None,
+             ld_pad=0):
+    """Encode + decode on the GPU and with the oracle; returns both result sets."""
+    from paper_2605_15890_b200.session import Session
+    rp, ci, a, w = code
+    k = G_host.shape[0]
+    d = G_host.shape[1] if d is None else d
+    n = len(bits)
+    if any(b == 1 for b in bits):
+        flags |= agc.AGC_FLAG_ALLOW_1BIT
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=seed, flags=flags | agc.AGC_FLAG_NO_UNBIASED_CHECK)
+    ld = ((d + 3) // 4) * 4 + ld_pad
+    G = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+    G[:, :d] = torch.from_numpy(np.ascontiguousarray(G_host[:, :d]))
+    if ld > d:
+        G[:, d:] = 7.0  # padding the kernel must never read as data
+    ses.codes.fill_(-1)
+    ses.scales.fill_(-1.0)
+    ses.encode(G, rnd)
+    masks = np.atleast_2d(masks).astype(np.uint8)
+    R = masks.shape[0]
+    m_dev = torch.from_numpy(masks).cuda()
+    ghat = torch.full((R, d), -3.0, dtype=torch.float32, device="cuda")
+    ses.decode(m_dev, ghat=ghat)
+    out = dict(codes=ses.codes_host(), scales=ses.scales_host(), ghat=ghat.cpu().numpy(),
+               status=int(ses.status.item()), tma=ses.uses_tma)
+    if beta0 is not None:
+        b1 = torch.from_numpy(beta0.copy()).cuda()
+        ses.decode(m_dev, lr=lr, ghat=ghat, beta=b1)      # sequential definition
+        out["beta_seq"] = b1.cpu().numpy()
+        b2 = torch.from_numpy(beta0.copy()).cuda()
+        ses.decode(m_dev, lr=lr, beta=b2)                  # collapsed when R > 1
+        out["beta_fused"] = b2.cpu().numpy()
+    torch.cuda.synchronize()
+    ses.close()
+    oc, osc, ost, _ = orp.encode_quantize(rp, ci, a, bits, B, seed, rnd, G_host[:, :d], d=d)
+    og, ob = orp.decode(d, bits, B, w, masks, oc, osc, lr=lr, beta=beta0)
+    ref = dict(codes=oc, scales=osc, ghat=og, status=ost, beta=ob)
+    return out, ref
+
+
+def assert_exact(out, ref):
+    assert out["scales"].shape == ref["scales"].shape
+    assert (out["scales"].view(np.uint32) == ref["scales"].view(np.uint32)).all()
+    assert out["codes"].shape == ref["codes"].shape
+    bad = np.nonzero(out["codes"] != ref["codes"])[0]
+    assert bad.size == 0, f"{bad.size} code words differ, first at {bad[:5]}"
+    assert (out["ghat"].view(np.uint32) == ref["ghat"].view(np.uint32)).all()
+    assert (out["status"] & 1) == (ref["status"] & 1)
+    assert out["status"] & 4 == 0
+
+
+def test_config1_all_rounds_bit_exact(agc, torch):
+    """n=k=4, cyclic s=2, d=10,000 (not a multiple of the block), b=(2,3,4,8), 100 rounds
+    each with a fresh Bernoulli straggler mask."""
+    wl = cfgs.config1()
+    code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
+    masks = cfgs.straggler_masks(wl)
+    for t in range(wl.rounds):
+        G = cfgs.partials_numpy(wl, t)
+        out, ref = run_both(agc, torch, G, code, wl.p, wl.bits, 512, wl.seed, t, masks[t, 0])
+        assert_exact(out, ref)
+        assert out["tma"]
+
+
+@pytest.mark.parametrize("d", [1, 3, 127, 128, 129, 511, 512, 513, 1000, 4097, 70001])
+@pytest.mark.parametrize("B", [128, 256, 512])
+@pytest.mark.parametrize("direct", [False, True])
+def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
+    rng = np.random.default_rng(d * 7 + B)
+    n = k = 8
+    bits = np.arange(1, 9, dtype=np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    code = _codes.cyclic_code(p, bits, k, 3, B)
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-3, 2, (k, 1))).astype(np.float32)
+    masks = (rng.random((2, n)) > 0.3).astype(np.uint8)
+    out, ref = run_both(agc, torch, G, code, p, bits, B, 1234 + d, 5, masks,
+                        flags=agc.AGC_FLAG_FORCE_DIRECT if direct else 0, ld_pad=4 if d % 2 else 0)
+    assert_exact(out, ref)
+    assert out["tma"] == (not direct)
+
+
+@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups"])
+def test_code_structures(agc, torch, kind):
+    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups"].index(kind))
+    d = 3000
+    if kind == "identity":
+        n = k = 5
+        bits = np.array([2, 8, 3, 5, 4], np.uint8)
+        p = np.zeros(n)
+        code = _codes.identity_code(n)
+    elif kind == "interval":
+        n, k = 7, 12
+        bits = rng.integers(2, 9, n).astype(np.uint8)
+        p = rng.uniform(0.05, 0.5, n)
+        code = _codes.interval_code(p, bits, k, 512)
+    elif kind == "s1":
+        n = k = 6
+        bits = rng.integers(2, 9, n).astype(np.uint8)
+        p = rng.uniform(0.05, 0.5, n)
+        code = _codes.cyclic_code(p, bits, k, 1, 512)
+    elif kind == "s_eq_k":
+        n = k = 6
+        bits = rng.integers(2, 9, n).astype(np.uint8)
+        p = rng.uniform(0.05, 0.5, n)
+        code = _codes.cyclic_code(p, bits, k, k, 512)
+    elif kind == "wide_rows":      # a support wider than a staged tile: direct kernel
+        n, k = 3, 50
+        bits = np.array([4, 6, 8], np.uint8)
+        p = rng.uniform(0.05, 0.5, n)
+        code = _codes.cyclic_code(p, bits, k, 40, 512)
+    else:                          # many worker groups per block in the staged kernel
+        n = k = 100
+        bits = rng.integers(1, 9, n).astype(np.uint8)
+        p = rng.uniform(0.01, 0.6, n)
+        code = _codes.cyclic_code(p, bits, k, 5, 512)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    masks = (rng.random((1, n)) >= p).astype(np.uint8)
+    out, ref = run_both(agc, torch, G, code, p, bits, 512, 77, 3, masks)
+    assert_exact(out, ref)
+    assert out["tma"] == (kind != "wide_rows")
+
+
+def test_straggler_extremes_and_batched_decode(agc, torch):
+    """All stragglers (g_hat = 0), none, single survivors; R realisations with per-
+    realisation outputs, the sequential update and the collapsed update."""
+    rng = np.random.default_rng(11)
+    n = k = 8
+    d = 5000
+    bits = np.array([1, 2, 3, 4, 5, 6, 7, 8], np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    code = _codes.cyclic_code(p, bits, k, 2, 256)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    masks = np.concatenate([np.zeros((1, n)), np.ones((1, n)), np.eye(n), rng.random((6, n)) > 0.4]).astype(np.uint8)
+    R = masks.shape[0]
+    lr = rng.uniform(0.001, 0.01, R).astype(np.float32)
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    out, ref = run_both(agc, torch, G, code, p, bits, 256, 3, 9, masks, lr=lr, beta0=beta0)
+    assert_exact(out, ref)
+    assert (out["ghat"][0] == 0).all()
+    assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
+    rel = np.abs(out["beta_fused"] - ref["beta"]).max() / np.abs(ref["beta"]).max()
+    assert rel <= 1e-5
+    # R = 1 fused update is the definition itself
+    out1, ref1 = run_both(agc, torch, G, code, p, bits, 256, 3, 9, masks[12:13], lr=lr[:1], beta0=beta0)
+    assert (out1["beta_fused"].view(np.uint32) == ref1["beta"].view(np.uint32)).all()
+
+
+def test_nonfinite_and_zero_buckets(agc, torch):
+    rng = np.random.default_rng(2)
+    n = k = 4
+    d = 2048
+    bits = np.array([1, 2, 5, 8], np.uint8)
+    p = np.full(n, 0.2)
+    code = _codes.cyclic_code(p, bits, k, 2, 512)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    G[:, 512:1024] = 0.0
+    G[1, 1500] = np.inf
+    G[2, 100] = np.nan
+    out, ref = run_both(agc, torch, G, code, p, bits, 512, 1, 0, np.ones((1, n)))
+    assert ref["status"] & 1 and out["status"] & 1
+    assert (out["scales"].view(np.uint32) == ref["scales"].view(np.uint32)).all()
+    assert (out["codes"] == ref["codes"]).all()
+    both_nan = np.isnan(out["ghat"]) & np.isnan(ref["ghat"])
+    assert ((out["ghat"].view(np.uint32) == ref["ghat"].view(np.uint32)) | both_nan).all()
+
+
+def test_same_round_same_bits_other_round_other_bits(agc, torch):
+    wl = cfgs.config1()
+    code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
+    G = cfgs.partials_numpy(wl, 0)
+    a, _ = run_both(agc, torch, G, code, wl.p, wl.bits, 512, 5, 7, np.ones((1, 4)))
+    b, _ = run_both(agc, torch, G, code, wl.p, wl.bits, 512, 5, 7, np.ones((1, 4)))
+    c, _ = run_both(agc, torch, G, code, wl.p, wl.bits, 512, 5, 8, np.ones((1, 4)))
+    assert (a["codes"] == b["codes"]).all() and (a["codes"] != c["codes"]).any()
+
+
+def test_config2_rounds_bit_exact(agc, torch):
+    """n=k=16, s=3, d=2^20, per-partition scales log-uniform in [1e-3, 1], bits from the
+    allocator under Z_tot = 64."""
+    wl = cfgs.config2()
+    bits, _ = od.bit_allocate_low_complexity(wl.p, wl.z_tot, 512, b_max=8)
+    code = _codes.cyclic_code(wl.p, bits, wl.k, wl.s, 512)
+    masks = cfgs.straggler_masks(wl, rounds=2)
+    for t in range(2):
+        G = cfgs.partials_numpy(wl, t)
+        out, ref = run_both(agc, torch, G, code, wl.p, bits, 512, wl.seed, t, masks[t, 0])
+        assert_exact(out, ref)
+
+
+def test_host_buffer_round(agc, torch):
+    from paper_2605_15890_b200.session import Session
+    wl = cfgs.config1()
+    rp, ci, a, w = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
+    ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, wl.bits, bucket=512, seed=3)
+    G = torch.from_numpy(cfgs.partials_numpy(wl, 0)).pin_memory()
+    mask = torch.tensor([1, 0, 1, 1], dtype=torch.uint8).pin_memory()
+    ghat = torch.empty(wl.d, dtype=torch.float32).pin_memory()
+    for rnd in (0, 1):
+        st = agc.agc_round_host(ses.plan, G, wl.d, rnd, mask, ghat)
+        assert st == 0
+        oc, osc, _, _ = orp.encode_quantize(rp, ci, a, wl.bits, 512, 3, rnd, G.numpy())
+        og, _ = orp.decode(wl.d, wl.bits, 512, w, mask.numpy()[None], oc, osc)
+        assert (ghat.numpy().view(np.uint32) == og[0].view(np.uint32)).all()
+    ses.close()
