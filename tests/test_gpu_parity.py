@@ -131,8 +131,8 @@ def test_code_structures(agc, torch, kind):
         p = rng.uniform(0.05, 0.5, n)
         code = _codes.cyclic_code(p, bits, k, k, 512)
     elif kind == "wide_rows":      # a support wider than a staged tile: direct kernel
-        n, k = 3, 50
-        bits = np.array([4, 6, 8], np.uint8)
+        n = k = 45
+        bits = rng.integers(2, 9, n).astype(np.uint8)
         p = rng.uniform(0.05, 0.5, n)
         code = _codes.cyclic_code(p, bits, k, 40, 512)
     else:                          # many worker groups per block in the staged kernel
