@@ -52,6 +52,7 @@ extern "C" {
 #define AGC_ERR_STATE (-7)      /* plan cannot serve this call (e.g. R too large)       */
 #define AGC_ERR_BUDGET (-8)     /* bit budget infeasible for the allocator              */
 #define AGC_ERR_NOMEM (-9)      /* host or device allocation failed                     */
+#define AGC_ERR_LIMIT (-10)     /* size beyond a fixed limit of agc_decode_update_static */
 
 #define AGC_FLAG_ALLOW_1BIT 1u         /* accept b_i = 1 (two-point quantiser; outside the paper)  */
 #define AGC_FLAG_NO_UNBIASED_CHECK 2u  /* skip the check of the unbiasedness condition             */
@@ -148,6 +149,45 @@ int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64
 int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
                const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
                float *beta_dev, void *cuda_stream);
+
+/*
+ * agc_decode_update_static - the multi-realisation fused update without any allocation.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - a training
+ * process whose device memory was handed over in full to a framework's pool at
+ * start-up, a plug-in that is given buffers and must not grow the process's footprint,
+ * a latency-critical loop that cannot take the device-wide synchronisation cudaMalloc
+ * and cudaFree imply. Such callers cannot build a plan (agc_plan_create allocates the
+ * plan's device tables), so this call takes the per-worker tables from the host and
+ * keeps its working data - the tables, the learning rates and the effective weights
+ * sum_r lr_r I_{r,i} - in a fixed array that is part of the library image on every GPU
+ * that loads it (about 33 KiB per GPU, held until the process exits). It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Computes, like agc_decode with R realisations, beta_dev only:
+ *   beta <- beta - sum_i (sum_r lr_r I_{r,i}) w_i q_i
+ *
+ *   n_workers  1..1024;  d  as in agc_plan_create;  bucket  128, 256 or 512
+ *   bits, w    host, n entries each: b_i in 1..8 and the decoding coefficients w_i
+ *   codes_dev, scales_dev  device, laid out as agc_encode_quantize writes them for the
+ *              same (n, d, bits, bucket); codes_dev 16-byte aligned
+ *   masks_dev  device, R x n bytes, 1 = arrived
+ *   R          1..4096;  lr_host  host, R learning rates
+ *   beta_dev   device in/out, d fp32, 16-byte aligned
+ * Returns AGC_ERR_LIMIT when n_workers or R exceeds the limits above (nothing is
+ * launched), otherwise as agc_decode. Asynchronous on the stream.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture. All calls on a device
+ * share the one array: each call rewrites every entry it later reads, so nothing has
+ * to be cleared between calls, but two calls whose GPU work overlaps (different
+ * streams, or different threads) race on it - keep them on one stream or order them.
+ */
+int agc_decode_update_static(int n_workers, int64_t d, uint32_t bucket, const uint8_t *bits,
+                             const float *w, const void *codes_dev, const float *scales_dev,
+                             const uint8_t *masks_dev, int R, const float *lr_host,
+                             float *beta_dev, void *cuda_stream);
 
 /*
  * agc_round_host - a whole round through host buffers: copies G to the device,

@@ -19,6 +19,7 @@ AGC_STATUS_NONFINITE = 1
 AGC_STATUS_TIMEOUT = 4
 AGC_CODE_INTERVAL = 0
 AGC_CODE_SUPPORT = 1
+AGC_ERR_LIMIT = -10
 
 
 class AgcError(RuntimeError):
@@ -56,6 +57,9 @@ def _load():
     L.agc_encode_quantize.restype = C.c_int
     L.agc_decode.argtypes = [vp, vp, vp, vp, C.c_int, f32p, vp, vp, vp]
     L.agc_decode.restype = C.c_int
+    L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
+                                           vp, vp]
+    L.agc_decode_update_static.restype = C.c_int
     L.agc_round_host.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, u32p, vp]
     L.agc_round_host.restype = C.c_int
     for name in ("agc_bit_allocate", "agc_bit_allocate_dp"):
@@ -160,6 +164,18 @@ def agc_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host=None, ghat_dev
         raise AgcError(-1, "lr_host shorter than R")
     _check(_lib.agc_decode(plan, _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
                            _hp(lr, C.c_float), _dev(ghat_dev), _dev(beta_dev), _stream(stream)))
+
+
+def agc_decode_update_static(n_workers, d, bucket, bits, w, codes_dev, scales_dev, masks_dev, R, lr_host,
+                             beta_dev, stream=None):
+    """Multi-realisation fused update that allocates nothing (its scratch is a fixed array
+    inside the library). bits / w / lr_host are host arrays; the rest are device buffers."""
+    bits, w, lr = _np(bits, np.uint8), _np(w, np.float32), _np(lr_host, np.float32)
+    if len(bits) != n_workers or len(w) != n_workers or lr.size < R:
+        raise AgcError(-1, "array lengths do not match n_workers / R")
+    _check(_lib.agc_decode_update_static(n_workers, d, bucket, _hp(bits, C.c_uint8), _hp(w, C.c_float),
+                                         _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
+                                         _hp(lr, C.c_float), _dev(beta_dev), _stream(stream)))
 
 
 def agc_round_host(plan, G_host, ld_host, rnd, mask_host, ghat_host, stream=None):

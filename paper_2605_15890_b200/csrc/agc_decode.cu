@@ -5,6 +5,8 @@
 // One warp owns one 512-coordinate pack block. Lane l holds the 16 coordinates
 // {128c + 4l + e}, i.e. stream positions 16l..16l+15 of every worker's message, so it
 // reads 16*b_i contiguous bits per worker and never needs another lane's data.
+#include <mutex>
+
 #include "agc_internal.h"
 
 namespace {
@@ -221,5 +223,104 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     } else {
         launch<false>(P, grid, stream);
     }
+    return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ allocation-free update
+// Multi-realisation fused update for callers that must not allocate device memory: the
+// per-worker tables and the effective weights live in one static device array that
+// every GPU loading the library carries until the process exits.
+#define AGC_STATIC_MAX_DEVICES 64
+
+namespace {
+
+struct AgcStaticScratch {
+    long long word_off[AGC_STATIC_MAX_WORKERS + 1];
+    float weff[AGC_STATIC_MAX_WORKERS];
+    float w[AGC_STATIC_MAX_WORKERS];
+    float lr[AGC_STATIC_MAX_R];
+    uint8_t bits[AGC_STATIC_MAX_WORKERS];
+};
+
+}  // namespace
+
+// In host code this name is only a handle for the runtime's symbol calls, never an
+// address a kernel may be given; agc_static_scratch_address() resolves it per device.
+static __device__ __align__(256) unsigned char agc_static_scratch[sizeof(AgcStaticScratch)];
+
+namespace {
+
+std::mutex g_static_mu;
+void *g_static_ptr[AGC_STATIC_MAX_DEVICES] = {};
+
+// Device address of the scratch array on the current device, looked up once per device.
+int agc_static_scratch_address(AgcStaticScratch **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AGC_ERR_CUDA;
+    if (dev < 0 || dev >= AGC_STATIC_MAX_DEVICES) return AGC_ERR_LIMIT;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, agc_static_scratch) != cudaSuccess || !ptr) return AGC_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = static_cast<AgcStaticScratch *>(g_static_ptr[dev]);
+    return AGC_OK;
+}
+
+}  // namespace
+
+extern "C" int agc_decode_update_static(int n_workers, int64_t d, uint32_t bucket, const uint8_t *bits,
+                                        const float *w, const void *codes_dev, const float *scales_dev,
+                                        const uint8_t *masks_dev, int R, const float *lr_host,
+                                        float *beta_dev, void *cuda_stream)
+{
+    if (n_workers < 1 || d < 1 || d > (int64_t(1) << 31) - 1024 || R < 1) return AGC_ERR_ARG;
+    if (!bits || !w || !codes_dev || !scales_dev || !masks_dev || !lr_host || !beta_dev) return AGC_ERR_ARG;
+    if (bucket != 128 && bucket != 256 && bucket != 512) return AGC_ERR_ARG;
+    if (n_workers > AGC_STATIC_MAX_WORKERS || R > AGC_STATIC_MAX_R) return AGC_ERR_LIMIT;
+    if ((reinterpret_cast<uintptr_t>(codes_dev) & 15) || (reinterpret_cast<uintptr_t>(beta_dev) & 15))
+        return AGC_ERR_ALIGN;
+    for (int i = 0; i < n_workers; ++i)
+        if (bits[i] < 1 || bits[i] > 8) return AGC_ERR_BITS;
+
+    AgcStaticScratch *sc = nullptr;
+    const int rc = agc_static_scratch_address(&sc);
+    if (rc != AGC_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const long long nblk = (d + AGC_BLOCK - 1) / AGC_BLOCK;
+    long long word_off[AGC_STATIC_MAX_WORKERS + 1];
+    word_off[0] = 0;
+    for (int i = 0; i < n_workers; ++i) word_off[i + 1] = word_off[i] + nblk * 16 * bits[i];
+    // every table entry a kernel of this call reads is rewritten here, so nothing left
+    // behind by an earlier call (same or different sizes) is ever used
+    if (cudaMemcpyAsync(sc->word_off, word_off, sizeof(long long) * (n_workers + 1), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(sc->w, w, sizeof(float) * n_workers, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(sc->bits, bits, n_workers, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(sc->lr, lr_host, sizeof(float) * R, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return AGC_ERR_CUDA;
+
+    AgcDecParams P;
+    P.bits = sc->bits;
+    P.w = sc->w;
+    P.word_off = sc->word_off;
+    P.codes = static_cast<const uint32_t *>(codes_dev);
+    P.scales = scales_dev;
+    P.masks = masks_dev;
+    P.weff = sc->weff;
+    P.ghat = nullptr;
+    P.beta = beta_dev;
+    P.d = d;
+    P.nblk = nblk;
+    P.nb = (d + bucket - 1) / bucket;
+    P.n = n_workers;
+    P.R = R;
+    P.rows_per_bucket = int(bucket) / 128;
+    P.lr0 = 0.0f;
+    P.lr = sc->lr;
+    agc_effective_weights_kernel<<<(n_workers + 127) / 128, 128, 0, stream>>>(masks_dev, sc->lr, n_workers, R, sc->weff);
+    launch<true>(P, (int)((nblk + 7) / 8), stream);
     return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
 }

@@ -13,6 +13,8 @@
 #define AGC_MAX_STAGE_ROWS 36  // partition rows per staged tile (36 * 2 KiB = 72 KiB)
 #define AGC_ENC_CONSUMER_WARPS 16
 #define AGC_MAX_R 4096         // straggler realisations per decode call
+#define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
+#define AGC_STATIC_MAX_R 4096
 
 // Parameters of one encode launch (passed by value; lives in the constant bank).
 struct AgcEncParams {

@@ -268,6 +268,7 @@ extern "C" const char *agc_strerror(int code)
         case AGC_ERR_STATE: return "plan cannot serve this call";
         case AGC_ERR_BUDGET: return "bit budget infeasible";
         case AGC_ERR_NOMEM: return "out of memory";
+        case AGC_ERR_LIMIT: return "size beyond the fixed limit of the allocation-free entry point";
         default: return "unknown error";
     }
 }
