@@ -11,10 +11,26 @@
 #define AGC_FRAC_BITS 15       // fractional bits of the fixed-point stochastic rounding
 #define AGC_MAX_STAGES 16      // shared-memory ring depth limit of the staged encoder
 #define AGC_MAX_STAGE_ROWS 36  // partition rows per staged tile (36 * 2 KiB = 72 KiB)
+#ifndef AGC_ENC_CONSUMER_WARPS
 #define AGC_ENC_CONSUMER_WARPS 16
+#endif
+#define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
 #define AGC_MAX_R 4096         // straggler realisations per decode call
 #define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
 #define AGC_STATIC_MAX_R 4096
+
+// Per-worker and per-entry records of the staged encoder (copied to shared memory).
+struct __align__(16) AgcWorkerDesc {
+    long long word_off;   // word offset of the worker's message
+    uint32_t e0;          // first entry of the worker's row of A
+    uint16_t ne;          // entries in that row
+    uint8_t bits;
+    uint8_t pad;
+};
+struct __align__(8) AgcEntryDesc {
+    float a;              // coefficient a_ij
+    uint32_t off;         // byte offset of partition row j inside its group's staged tile
+};
 
 // Parameters of one encode launch (passed by value; lives in the constant bank).
 struct AgcEncParams {
@@ -22,7 +38,8 @@ struct AgcEncParams {
     const int32_t *col_idx;      // nnz
     const float *a;              // nnz
     const uint8_t *bits;         // n
-    const uint8_t *ent_slot;     // nnz: slot of entry's partition row inside its group's tile
+    const AgcWorkerDesc *wdesc;  // n
+    const AgcEntryDesc *edesc;   // nnz
     const long long *word_off;   // n+1: word offset of each worker's message
     const int32_t *grp_row_ptr;  // n_groups+1
     const int32_t *grp_rows;     // partition row per tile slot
@@ -33,7 +50,7 @@ struct AgcEncParams {
     float *scales;
     uint32_t *status;
     long long d, ld, nblk, nb;
-    int n, k, n_groups;
+    int n, k, n_groups, nnz;
     int rows_per_bucket;         // bucket / 128: 1, 2 or 4
     int stages, stage_rows;
     uint32_t round_lo, round_hi;
@@ -75,7 +92,9 @@ struct agc_plan {
     // device tables
     int32_t *d_row_ptr = nullptr, *d_col_idx = nullptr;
     float *d_a = nullptr, *d_w = nullptr;
-    uint8_t *d_bits = nullptr, *d_ent_slot = nullptr;
+    uint8_t *d_bits = nullptr;
+    AgcWorkerDesc *d_wdesc = nullptr;
+    AgcEntryDesc *d_edesc = nullptr;
     long long *d_word_off = nullptr;
     int32_t *d_grp_row_ptr = nullptr, *d_grp_rows = nullptr, *d_grp_wk_ptr = nullptr, *d_grp_workers = nullptr;
     // decode scratch

@@ -1,4 +1,5 @@
 // Plan object, argument validation, size queries and the host-buffer round.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -62,7 +63,7 @@ bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::ve
 void free_device(agc_plan *p)
 {
     cudaFree(p->d_row_ptr); cudaFree(p->d_col_idx); cudaFree(p->d_a); cudaFree(p->d_w);
-    cudaFree(p->d_bits); cudaFree(p->d_ent_slot); cudaFree(p->d_word_off);
+    cudaFree(p->d_bits); cudaFree(p->d_wdesc); cudaFree(p->d_edesc); cudaFree(p->d_word_off);
     cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_rows); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
     cudaFree(p->d_weff); cudaFree(p->d_lr);
     cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
@@ -138,8 +139,23 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     bool stageable = build_groups(*pl, grp_row_ptr, grp_rows, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
     pl->n_groups = int(grp_row_ptr.size()) - 1;
     pl->use_tma = false;
-    if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0) {
-        const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16;
+    std::vector<AgcWorkerDesc> wdesc(n_workers);
+    std::vector<AgcEntryDesc> edesc(nnz);
+    for (int i = 0; i < n_workers; ++i) {
+        wdesc[i].word_off = pl->word_off[i];
+        wdesc[i].e0 = uint32_t(row_ptr[i]);
+        wdesc[i].ne = uint16_t(std::min(row_ptr[i + 1] - row_ptr[i], 65535));
+        wdesc[i].bits = bits[i];
+        wdesc[i].pad = 0;
+    }
+    for (int e = 0; e < nnz; ++e) {
+        edesc[e].a = a[e];
+        edesc[e].off = stageable ? uint32_t(ent_slot[e]) * AGC_BLOCK * sizeof(float) : 0u;
+    }
+    const size_t table_bytes = sizeof(AgcWorkerDesc) * n_workers + sizeof(AgcEntryDesc) * nnz +
+                               sizeof(int32_t) * (size_t(pl->n_groups) + 1 + n_workers) + 16;
+    if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0 && table_bytes <= AGC_ENC_TABLE_BYTES_MAX) {
+        const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16 + table_bytes;
         const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);
         long long stages = (long long)((size_t(smem_optin) - tail - 1024) / stage_bytes);
         if (stages > AGC_MAX_STAGES) stages = AGC_MAX_STAGES;
@@ -161,7 +177,8 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc) rc = upload(&pl->d_a, pl->a);
     if (!rc) rc = upload(&pl->d_w, pl->w);
     if (!rc) rc = upload(&pl->d_bits, pl->bits);
-    if (!rc) rc = upload(&pl->d_ent_slot, ent_slot);
+    if (!rc) rc = upload(&pl->d_wdesc, wdesc);
+    if (!rc) rc = upload(&pl->d_edesc, edesc);
     if (!rc) rc = upload(&pl->d_word_off, pl->word_off);
     if (!rc) rc = upload(&pl->d_grp_row_ptr, grp_row_ptr);
     if (!rc) rc = upload(&pl->d_grp_rows, grp_rows);
