@@ -12,7 +12,7 @@
 #define AGC_MAX_STAGES 16      // shared-memory ring depth limit of the staged encoder
 #define AGC_MAX_STAGE_ROWS 36  // partition rows per staged tile (36 * 2 KiB = 72 KiB)
 #ifndef AGC_ENC_CONSUMER_WARPS
-#define AGC_ENC_CONSUMER_WARPS 16
+#define AGC_ENC_CONSUMER_WARPS 23  // + 1 producer warp = 6 warps per scheduler at 80 registers
 #endif
 #define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
 #define AGC_MAX_R 4096         // straggler realisations per decode call
@@ -21,16 +21,27 @@
 
 // Per-worker and per-entry records of the staged encoder (copied to shared memory).
 struct __align__(16) AgcWorkerDesc {
-    long long word_off;   // word offset of the worker's message
-    uint32_t e0;          // first entry of the worker's row of A
-    uint16_t ne;          // entries in that row
+    long long word_off;    // word offset of the worker's message
+    long long scales_off;  // element offset of the worker's row of scales: i * nb
+    uint32_t e0;           // first entry of the worker's row of A
+    uint16_t ne;           // entries in that row
     uint8_t bits;
     uint8_t pad;
+    uint32_t pad2[2];
 };
 struct __align__(8) AgcEntryDesc {
     float a;              // coefficient a_ij
     uint32_t off;         // byte offset of partition row j inside its group's staged tile
 };
+
+// One TMA box of a staged tile: partition rows [row, row + (32 >> hsel)) go to the
+// tile's row slots starting at `slot` (both 256-column halves).
+struct AgcLoadOp {
+    uint16_t slot;
+    uint16_t hsel;
+    int32_t row;
+};
+#define AGC_ENC_BOX_SIZES 6  // box heights 32, 16, 8, 4, 2, 1
 
 // Parameters of one encode launch (passed by value; lives in the constant bank).
 struct AgcEncParams {
@@ -41,8 +52,9 @@ struct AgcEncParams {
     const AgcWorkerDesc *wdesc;  // n
     const AgcEntryDesc *edesc;   // nnz
     const long long *word_off;   // n+1: word offset of each worker's message
-    const int32_t *grp_row_ptr;  // n_groups+1
-    const int32_t *grp_rows;     // partition row per tile slot
+    const int32_t *grp_row_ptr;  // n_groups+1: rows (tile slots) of each group
+    const int32_t *grp_op_ptr;   // n_groups+1
+    const AgcLoadOp *ops;        // TMA boxes of each group's tile
     const int32_t *grp_wk_ptr;   // n_groups+1
     const int32_t *grp_workers;  // workers of each group
     const float *G;
@@ -51,7 +63,6 @@ struct AgcEncParams {
     uint32_t *status;
     long long d, ld, nblk, nb;
     int n, k, n_groups, nnz;
-    int rows_per_bucket;         // bucket / 128: 1, 2 or 4
     int stages, stage_rows;
     uint32_t round_lo, round_hi;
     uint32_t rk[20];             // Philox round keys: rk[2r] = key0 + r*W0, rk[2r+1] = key1 + r*W1
@@ -96,7 +107,8 @@ struct agc_plan {
     AgcWorkerDesc *d_wdesc = nullptr;
     AgcEntryDesc *d_edesc = nullptr;
     long long *d_word_off = nullptr;
-    int32_t *d_grp_row_ptr = nullptr, *d_grp_rows = nullptr, *d_grp_wk_ptr = nullptr, *d_grp_workers = nullptr;
+    int32_t *d_grp_row_ptr = nullptr, *d_grp_op_ptr = nullptr, *d_grp_wk_ptr = nullptr, *d_grp_workers = nullptr;
+    AgcLoadOp *d_ops = nullptr;
     // decode scratch
     float *d_weff = nullptr, *d_lr = nullptr;
     // staging for the host-buffer entry point (allocated on first use)

@@ -21,25 +21,49 @@ int upload(T **dst, const std::vector<T> &src)
 }
 
 // Partition the workers (in order) into groups whose supports together touch at most
-// AGC_MAX_STAGE_ROWS partition rows: one staged tile = (pack block, group). Returns
-// false when some worker's own support is too wide for a tile.
-bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::vector<int32_t> &grp_rows,
-                  std::vector<int32_t> &grp_wk_ptr, std::vector<int32_t> &grp_workers,
-                  std::vector<uint8_t> &ent_slot, int *max_rows)
+// AGC_MAX_STAGE_ROWS partition rows: one staged tile = (pack block, group). Inside a tile
+// the rows sit in ascending partition order; each run of consecutive partitions is cut
+// into boxes of 32, 16, 8, 4, 2 or 1 rows. Returns false when some worker's own support
+// is too wide for a tile.
+bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::vector<int32_t> &grp_op_ptr,
+                  std::vector<AgcLoadOp> &ops, std::vector<int32_t> &grp_wk_ptr,
+                  std::vector<int32_t> &grp_workers, std::vector<uint16_t> &ent_slot, int *max_rows)
 {
     grp_row_ptr.assign(1, 0);
+    grp_op_ptr.assign(1, 0);
     grp_wk_ptr.assign(1, 0);
-    grp_rows.clear();
+    ops.clear();
     grp_workers.clear();
     ent_slot.assign(pl.col_idx.size(), 0);
+    std::vector<char> in_group(pl.k, 0);
     std::vector<int> slot_of(pl.k, -1);
     std::vector<int32_t> cur_rows;
     *max_rows = 0;
     auto flush = [&]() {
-        if (grp_workers.size() == size_t(grp_wk_ptr.back())) return;
-        for (int32_t r : cur_rows) { grp_rows.push_back(r); slot_of[r] = -1; }
-        grp_row_ptr.push_back(int32_t(grp_rows.size()));
-        grp_wk_ptr.push_back(int32_t(grp_workers.size()));
+        const int first = grp_wk_ptr.back(), last = int(grp_workers.size());
+        if (first == last) return;
+        std::sort(cur_rows.begin(), cur_rows.end());
+        for (size_t t = 0; t < cur_rows.size(); ++t) slot_of[cur_rows[t]] = int(t);
+        for (int wi = first; wi < last; ++wi) {
+            const int i = grp_workers[wi];
+            for (int e = pl.row_ptr[i]; e < pl.row_ptr[i + 1]; ++e) ent_slot[e] = uint16_t(slot_of[pl.col_idx[e]]);
+        }
+        for (size_t t = 0; t < cur_rows.size();) {
+            size_t u = t + 1;
+            while (u < cur_rows.size() && cur_rows[u] == cur_rows[u - 1] + 1) ++u;
+            size_t len = u - t;
+            while (len > 0) {
+                int hsel = 0;
+                while ((size_t(32) >> hsel) > len) ++hsel;
+                ops.push_back(AgcLoadOp{uint16_t(t), uint16_t(hsel), cur_rows[t]});
+                t += size_t(32) >> hsel;
+                len -= size_t(32) >> hsel;
+            }
+        }
+        for (int32_t r : cur_rows) in_group[r] = 0;
+        grp_row_ptr.push_back(grp_row_ptr.back() + int32_t(cur_rows.size()));
+        grp_op_ptr.push_back(int32_t(ops.size()));
+        grp_wk_ptr.push_back(last);
         *max_rows = std::max<int>(*max_rows, int(cur_rows.size()));
         cur_rows.clear();
     };
@@ -47,12 +71,11 @@ bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::ve
         const int e0 = pl.row_ptr[i], e1 = pl.row_ptr[i + 1];
         if (e1 - e0 > AGC_MAX_STAGE_ROWS) return false;
         int fresh = 0;
-        for (int e = e0; e < e1; ++e) fresh += slot_of[pl.col_idx[e]] < 0;
+        for (int e = e0; e < e1; ++e) fresh += !in_group[pl.col_idx[e]];
         if (int(cur_rows.size()) + fresh > AGC_MAX_STAGE_ROWS) flush();
         for (int e = e0; e < e1; ++e) {
             const int j = pl.col_idx[e];
-            if (slot_of[j] < 0) { slot_of[j] = int(cur_rows.size()); cur_rows.push_back(j); }
-            ent_slot[e] = uint8_t(slot_of[j]);
+            if (!in_group[j]) { in_group[j] = 1; cur_rows.push_back(j); }
         }
         grp_workers.push_back(i);
     }
@@ -64,7 +87,7 @@ void free_device(agc_plan *p)
 {
     cudaFree(p->d_row_ptr); cudaFree(p->d_col_idx); cudaFree(p->d_a); cudaFree(p->d_w);
     cudaFree(p->d_bits); cudaFree(p->d_wdesc); cudaFree(p->d_edesc); cudaFree(p->d_word_off);
-    cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_rows); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
+    cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_op_ptr); cudaFree(p->d_ops); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
     cudaFree(p->d_weff); cudaFree(p->d_lr);
     cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
     cudaFree(p->h_mask); cudaFree(p->h_status);
@@ -133,16 +156,19 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
         return AGC_ERR_CUDA;
     }
 
-    std::vector<int32_t> grp_row_ptr, grp_rows, grp_wk_ptr, grp_workers;
-    std::vector<uint8_t> ent_slot;
+    std::vector<int32_t> grp_row_ptr, grp_op_ptr, grp_wk_ptr, grp_workers;
+    std::vector<AgcLoadOp> ops;
+    std::vector<uint16_t> ent_slot;
     int max_rows = 0;
-    bool stageable = build_groups(*pl, grp_row_ptr, grp_rows, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
+    bool stageable = build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
     pl->n_groups = int(grp_row_ptr.size()) - 1;
     pl->use_tma = false;
     std::vector<AgcWorkerDesc> wdesc(n_workers);
     std::vector<AgcEntryDesc> edesc(nnz);
     for (int i = 0; i < n_workers; ++i) {
         wdesc[i].word_off = pl->word_off[i];
+        wdesc[i].scales_off = (long long)i * pl->nb;
+        wdesc[i].pad2[0] = wdesc[i].pad2[1] = 0;
         wdesc[i].e0 = uint32_t(row_ptr[i]);
         wdesc[i].ne = uint16_t(std::min(row_ptr[i + 1] - row_ptr[i], 65535));
         wdesc[i].bits = bits[i];
@@ -150,13 +176,13 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     }
     for (int e = 0; e < nnz; ++e) {
         edesc[e].a = a[e];
-        edesc[e].off = stageable ? uint32_t(ent_slot[e]) * AGC_BLOCK * sizeof(float) : 0u;
+        edesc[e].off = stageable ? uint32_t(ent_slot[e]) * 1024u : 0u;
     }
     const size_t table_bytes = sizeof(AgcWorkerDesc) * n_workers + sizeof(AgcEntryDesc) * nnz +
                                sizeof(int32_t) * (size_t(pl->n_groups) + 1 + n_workers) + 16;
     if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0 && table_bytes <= AGC_ENC_TABLE_BYTES_MAX) {
         const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16 + table_bytes;
-        const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);
+        const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);  // two halves of max_rows x 1 KiB
         long long stages = (long long)((size_t(smem_optin) - tail - 1024) / stage_bytes);
         if (stages > AGC_MAX_STAGES) stages = AGC_MAX_STAGES;
         cudaDriverEntryPointQueryResult qres;
@@ -181,7 +207,8 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc) rc = upload(&pl->d_edesc, edesc);
     if (!rc) rc = upload(&pl->d_word_off, pl->word_off);
     if (!rc) rc = upload(&pl->d_grp_row_ptr, grp_row_ptr);
-    if (!rc) rc = upload(&pl->d_grp_rows, grp_rows);
+    if (!rc) rc = upload(&pl->d_grp_op_ptr, grp_op_ptr);
+    if (!rc) rc = upload(&pl->d_ops, ops);
     if (!rc) rc = upload(&pl->d_grp_wk_ptr, grp_wk_ptr);
     if (!rc) rc = upload(&pl->d_grp_workers, grp_workers);
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
