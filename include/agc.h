@@ -139,6 +139,8 @@ int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64
  *   ghat_dev   device out or NULL: R x d fp32, realisation r at ghat_dev + r*d
  *   beta_dev   device in/out or NULL: d fp32 parameters, updated by
  *              beta <- beta - lr[r] * g_hat_r for r = 0..R-1
+ *   status_dev device, one uint32 or NULL: AGC_STATUS_TIMEOUT is OR-ed into it if a
+ *              bounded wait inside the kernel expired (outputs are then invalid)
  * With R = 1, or whenever ghat_dev is given, sums run over workers in ascending
  * order with fused multiply-adds (reproducible bit for bit). With R > 1 and only
  * beta_dev the R updates are applied in one pass through the linear form
@@ -148,7 +150,7 @@ int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64
  */
 int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
                const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
-               float *beta_dev, void *cuda_stream);
+               float *beta_dev, uint32_t *status_dev, void *cuda_stream);
 
 /*
  * agc_decode_update_static - the multi-realisation fused update without any allocation.

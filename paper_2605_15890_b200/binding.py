@@ -55,7 +55,7 @@ def _load():
     L.agc_plan_uses_tma.restype = C.c_int
     L.agc_encode_quantize.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, vp, vp]
     L.agc_encode_quantize.restype = C.c_int
-    L.agc_decode.argtypes = [vp, vp, vp, vp, C.c_int, f32p, vp, vp, vp]
+    L.agc_decode.argtypes = [vp, vp, vp, vp, C.c_int, f32p, vp, vp, vp, vp]
     L.agc_decode.restype = C.c_int
     L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
                                            vp, vp]
@@ -158,12 +158,13 @@ def agc_encode_quantize(plan, G_dev, ld, rnd, codes_dev, scales_dev, status_dev=
 
 
 def agc_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host=None, ghat_dev=None, beta_dev=None,
-               stream=None):
+               status_dev=None, stream=None):
     lr = None if lr_host is None else _np(lr_host, np.float32)
     if lr is not None and lr.size < R:
         raise AgcError(-1, "lr_host shorter than R")
     _check(_lib.agc_decode(plan, _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
-                           _hp(lr, C.c_float), _dev(ghat_dev), _dev(beta_dev), _stream(stream)))
+                           _hp(lr, C.c_float), _dev(ghat_dev), _dev(beta_dev), _dev(status_dev),
+                           _stream(stream)))
 
 
 def agc_decode_update_static(n_workers, d, bucket, bits, w, codes_dev, scales_dev, masks_dev, R, lr_host,

@@ -8,11 +8,19 @@
 #include <mutex>
 
 #include "agc_internal.h"
+#include "agc_ptx.cuh"
 
 namespace {
 
 // Add worker's contribution cstep[row] * level to the lane's 16 accumulators.
-template <int BITS>
+template <bool GLOBAL, typename T>
+__device__ __forceinline__ T load_words(const T *p)
+{
+    if constexpr (GLOBAL) return __ldg(p);
+    else return *p;
+}
+
+template <int BITS, bool GLOBAL = true>
 __device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int lane,
                                                   const float (&cstep_row)[4], float (&acc)[16])
 {
@@ -25,14 +33,14 @@ __device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int
         constexpr int NW = BITS / 2;
         const uint32_t *src = blk_words + lane * NW;
         if constexpr (NW == 4) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+            const uint4 v = load_words<GLOBAL>(reinterpret_cast<const uint4 *>(src));
             A[0] = v.x; A[1] = v.y; A[2] = v.z; A[3] = v.w;
         } else if constexpr (NW == 2) {
-            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+            const uint2 v = load_words<GLOBAL>(reinterpret_cast<const uint2 *>(src));
             A[0] = v.x; A[1] = v.y;
         } else {
 #pragma unroll
-            for (int t = 0; t < NW; ++t) A[t] = __ldg(src + t);
+            for (int t = 0; t < NW; ++t) A[t] = load_words<GLOBAL>(src + t);
         }
     } else {
         // a pair of lanes shares BITS words; the odd lane's slice starts at bit 16 of word H
@@ -40,7 +48,7 @@ __device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int
         const uint32_t *src = blk_words + (lane >> 1) * BITS + ((lane & 1) ? H : 0);
         uint32_t W[H + 1];
 #pragma unroll
-        for (int t = 0; t <= H; ++t) W[t] = __ldg(src + t);
+        for (int t = 0; t <= H; ++t) W[t] = load_words<GLOBAL>(src + t);
         if (lane & 1) {
 #pragma unroll
             for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
@@ -178,6 +186,218 @@ __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *
     weff[i] = s;
 }
 
+// ------------------------------------------------------------------ ring kernel
+// Persistent CTAs. A tile is AGC_DEC_QT consecutive pack blocks of one group of received
+// workers: the producer warp brings each worker's chunk (its words of those blocks are
+// contiguous in its message) into a shared-memory ring with one bulk copy, consumer warp
+// w unpacks block q0 + w of every worker of the group in ascending worker order. The
+// lane's 16 accumulators stay in registers across the groups of a tile row, so messages
+// of stragglers are never read and the summation order is the defining one.
+struct __align__(16) AgcDecWorker {
+    long long word_off;    // word offset of the worker's message
+    long long scales_off;  // i * nb
+    float weight;          // w_i, or w_i * (sum_r lr_r I_ri) in the collapsed mode
+    uint32_t soff;         // byte offset of the worker's chunk inside a stage
+    uint32_t bits;
+    uint32_t pad;
+};
+
+template <int BITS>
+__device__ __forceinline__ void ring_add_worker(const unsigned char *chunk, int warp, int lane,
+                                                const float (&ws_row)[4], float (&acc)[16])
+{
+    constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)((1 << (BITS >= 2 ? BITS - 1 : 1)) - 1)) : 2.0f;
+    float cstep_row[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
+    unpack_accumulate<BITS, false>(reinterpret_cast<const uint32_t *>(chunk) + warp * 16 * BITS, lane, cstep_row, acc);
+}
+
+template <int RB, bool COLLAPSED>
+__global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kernel(const AgcDecParams P)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int stages = P.stages;
+    const uint32_t stage_bytes = AGC_DEC_QT * 64u * AGC_DEC_GROUP_BITS;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)stages * stage_bytes);
+    uint64_t *empty = full + AGC_DEC_MAX_STAGES;
+    volatile int *flags = reinterpret_cast<volatile int *>(empty + AGC_DEC_MAX_STAGES);  // abort x2, n_groups
+    AgcDecWorker *s_wk = reinterpret_cast<AgcDecWorker *>(empty + AGC_DEC_MAX_STAGES + 2);
+    int32_t *s_grp_ptr = reinterpret_cast<int32_t *>(s_wk + P.n);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], AGC_DEC_QT);
+        }
+        flags[0] = 0;
+        flags[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async;" ::: "memory");
+        // compact list of the workers that contribute, cut into groups of at most 32 workers
+        // and AGC_DEC_GROUP_BITS bits per coordinate
+        int nrecv = 0, ng = 0, in_grp = 0;
+        uint32_t grp_bits = 0, soff = 0;
+        s_grp_ptr[0] = 0;
+        for (int i = 0; i < P.n; ++i) {
+            float wgt;
+            if (COLLAPSED) {
+                const float we = P.weff[i];
+                if (we == 0.0f) continue;
+                wgt = __fmul_rn(P.w[i], we);
+            } else {
+                if (!P.masks[i]) continue;
+                wgt = P.w[i];
+            }
+            const uint32_t b = P.bits[i];
+            if (in_grp == 32 || grp_bits + b > AGC_DEC_GROUP_BITS) {
+                s_grp_ptr[++ng] = nrecv;
+                in_grp = 0; grp_bits = 0; soff = 0;
+            }
+            AgcDecWorker wk;
+            wk.word_off = P.word_off[i];
+            wk.scales_off = (long long)i * P.nb;
+            wk.weight = wgt;
+            wk.soff = soff;
+            wk.bits = b;
+            wk.pad = 0;
+            s_wk[nrecv++] = wk;
+            soff += AGC_DEC_QT * 64u * b;
+            grp_bits += b;
+            ++in_grp;
+        }
+        if (in_grp) s_grp_ptr[++ng] = nrecv;
+        flags[2] = ng;
+    }
+    __syncthreads();
+    const int n_groups = flags[2];
+    const long long ntile = (P.nblk + AGC_DEC_QT - 1) / AGC_DEC_QT;
+
+    if (warp == AGC_DEC_QT) {
+        // ---------------- producer
+        long long issued = 0;
+        int s = 0;
+        uint32_t parity = 1;
+        bool ok = true;
+        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+            const long long q0 = T * AGC_DEC_QT;
+            const uint32_t nq = (uint32_t)(P.nblk - q0 < AGC_DEC_QT ? P.nblk - q0 : AGC_DEC_QT);
+            for (int g = 0; ok && g < n_groups; ++g) {
+                const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
+                uint32_t bytes = 0, soff = 0;
+                const unsigned char *src = nullptr;
+                if (lane < nr) {
+                    const AgcDecWorker wk = s_wk[r0 + lane];
+                    bytes = nq * 64u * wk.bits;
+                    soff = wk.soff;
+                    src = reinterpret_cast<const unsigned char *>(P.codes + wk.word_off + q0 * 16 * wk.bits);
+                }
+                uint32_t total = bytes;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+                ok = mbar_wait(&empty[s], parity, flags);
+                if (!ok) break;
+                if (lane == 0) mbar_arrive_expect_tx(&full[s], total);
+                __syncwarp();
+                if (lane < nr) bulk_load_1d(smem + (size_t)s * stage_bytes + soff, src, bytes, &full[s]);
+                ++issued;
+                if (++s == stages) { s = 0; parity ^= 1u; }
+            }
+        }
+        if (!ok) {
+            for (long long j = (issued > stages ? issued - stages : 0); j < issued; ++j)
+                mbar_wait(&full[j % stages], (uint32_t)((j / stages) & 1), flags + 1);
+        }
+    } else {
+        // ---------------- consumers: warp w owns pack block q0 + w of every tile
+        const bool vec = (P.d & 3) == 0;
+        int s = 0;
+        uint32_t parity = 0;
+        bool ok = true;
+        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+            const long long q = T * AGC_DEC_QT + warp;
+            const bool active = q < P.nblk;
+            float acc[16], b[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+            if (P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
+            for (int g = 0; ok && g < n_groups; ++g) {
+                const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
+                // the lane's worker of this group: its scale(s) for block q, fetched before the wait
+                float sc[4 / RB];
+#pragma unroll
+                for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
+                if (active && lane < nr) {
+                    const float *srow = P.scales + s_wk[r0 + lane].scales_off;
+#pragma unroll
+                    for (int bk = 0; bk < 4 / RB; ++bk) {
+                        const long long beta_idx = q * (4 / RB) + bk;
+                        if (beta_idx < P.nb) sc[bk] = __ldg(srow + beta_idx);
+                    }
+                }
+                ok = mbar_wait(&full[s], parity, flags);
+                if (!ok) break;
+                if (active) {
+                    const unsigned char *stage = smem + (size_t)s * stage_bytes;
+                    for (int r = 0; r < nr; ++r) {
+                        const AgcDecWorker wk = s_wk[r0 + r];
+                        float ws_row[4];
+#pragma unroll
+                        for (int bk = 0; bk < 4 / RB; ++bk) {
+                            const float S = __shfl_sync(0xffffffffu, sc[bk], r);
+                            const float ws = __fmul_rn(wk.weight, S);
+#pragma unroll
+                            for (int cc = 0; cc < RB; ++cc) ws_row[bk * RB + cc] = ws;
+                        }
+                        const unsigned char *chunk = stage + wk.soff;
+                        switch (wk.bits) {
+                            case 1: ring_add_worker<1>(chunk, warp, lane, ws_row, acc); break;
+                            case 2: ring_add_worker<2>(chunk, warp, lane, ws_row, acc); break;
+                            case 3: ring_add_worker<3>(chunk, warp, lane, ws_row, acc); break;
+                            case 4: ring_add_worker<4>(chunk, warp, lane, ws_row, acc); break;
+                            case 5: ring_add_worker<5>(chunk, warp, lane, ws_row, acc); break;
+                            case 6: ring_add_worker<6>(chunk, warp, lane, ws_row, acc); break;
+                            case 7: ring_add_worker<7>(chunk, warp, lane, ws_row, acc); break;
+                            default: ring_add_worker<8>(chunk, warp, lane, ws_row, acc); break;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[s]);
+                if (++s == stages) { s = 0; parity ^= 1u; }
+            }
+            if (ok && active) {
+                if (COLLAPSED) {
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) b[t] = __fsub_rn(b[t], acc[t]);
+                    store16(P.beta, q, lane, P.d, vec, b);
+                } else {
+                    if (P.ghat) store16(P.ghat, q, lane, P.d, vec, acc);
+                    if (P.beta) {
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) b[t] = __fmaf_rn(-P.lr0, acc[t], b[t]);
+                        store16(P.beta, q, lane, P.d, vec, b);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && (flags[0] || flags[1]) && P.status) atomicOr(P.status, AGC_STATUS_TIMEOUT);
+}
+
+template <bool COLLAPSED>
+cudaError_t launch_ring(const AgcDecParams &P, int grid, size_t smem, cudaStream_t stream)
+{
+    const int threads = (AGC_DEC_QT + 1) * 32;
+    if (P.rows_per_bucket == 4) agc_decode_ring_kernel<4, COLLAPSED><<<grid, threads, smem, stream>>>(P);
+    else if (P.rows_per_bucket == 2) agc_decode_ring_kernel<2, COLLAPSED><<<grid, threads, smem, stream>>>(P);
+    else agc_decode_ring_kernel<1, COLLAPSED><<<grid, threads, smem, stream>>>(P);
+    return cudaGetLastError();
+}
+
 template <bool COLLAPSED>
 void launch(const AgcDecParams &P, int grid, cudaStream_t stream)
 {
@@ -189,7 +409,8 @@ void launch(const AgcDecParams &P, int grid, cudaStream_t stream)
 }  // namespace
 
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
-                      int R, const float *lr_host, float *ghat, float *beta, cudaStream_t stream)
+                      int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
+                      cudaStream_t stream)
 {
     AgcDecParams P;
     P.bits = plan->d_bits;
@@ -209,7 +430,8 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     P.rows_per_bucket = plan->bucket / 128;
     P.lr0 = (beta && lr_host) ? lr_host[0] : 0.0f;
     P.lr = plan->d_lr;
-    const int grid = (int)((plan->nblk + 7) / 8);
+    P.status = status;
+    P.stages = plan->dec_stages;
     const bool collapsed = R > 1 && beta && !ghat;
     if (beta && R > 1) {
         if (cudaMemcpyAsync(plan->d_lr, lr_host, sizeof(float) * R, cudaMemcpyHostToDevice, stream) != cudaSuccess)
@@ -219,11 +441,52 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
         agc_effective_weights_kernel<<<(plan->n + 127) / 128, 128, 0, stream>>>(masks, plan->d_lr, plan->n, R,
                                                                                plan->d_weff);
         P.weff = plan->d_weff;
-        launch<true>(P, grid, stream);
-    } else {
-        launch<false>(P, grid, stream);
     }
+    if (plan->dec_ring) {
+        const long long ntile = (plan->nblk + AGC_DEC_QT - 1) / AGC_DEC_QT;
+        const int grid = (int)(ntile < plan->sm_count ? ntile : plan->sm_count);
+        if (collapsed) {
+            if (launch_ring<true>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
+        } else {
+            // one launch per realisation, in order: realisation r sees beta after r - 1
+            for (int r = 0; r < R; ++r) {
+                P.masks = masks + (size_t)r * plan->n;
+                P.ghat = ghat ? ghat + (size_t)r * plan->d : nullptr;
+                P.lr0 = (beta && lr_host) ? lr_host[r] : 0.0f;
+                if (launch_ring<false>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
+            }
+        }
+        return AGC_OK;
+    }
+    const int grid = (int)((plan->nblk + 7) / 8);
+    if (collapsed) launch<true>(P, grid, stream);
+    else launch<false>(P, grid, stream);
     return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
+}
+
+// Decide whether the plan decodes with the ring kernel and size its shared memory.
+int agc_decode_prepare(agc_plan *plan, int smem_optin)
+{
+    plan->dec_ring = false;
+    if ((plan->flags & AGC_FLAG_FORCE_DIRECT) || plan->n > AGC_DEC_RING_MAX_WORKERS) return AGC_OK;
+    const size_t stage_bytes = size_t(AGC_DEC_QT) * 64 * AGC_DEC_GROUP_BITS;
+    const size_t tail = (2 * AGC_DEC_MAX_STAGES + 2) * sizeof(uint64_t) + sizeof(AgcDecWorker) * size_t(plan->n) +
+                        sizeof(int32_t) * (size_t(plan->n) + 1) + 16;
+    if (size_t(smem_optin) < tail + 2 * stage_bytes) return AGC_OK;
+    long long stages = (long long)((size_t(smem_optin) - tail) / stage_bytes);
+    if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
+    plan->dec_stages = int(stages);
+    plan->dec_smem = size_t(stages) * stage_bytes + tail;
+    const int smem = int(plan->dec_smem);
+    if (cudaFuncSetAttribute(agc_decode_ring_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_ring_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_ring_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_ring_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_ring_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_ring_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    plan->dec_ring = true;
+    return AGC_OK;
 }
 
 // ------------------------------------------------------------------ allocation-free update

@@ -16,6 +16,14 @@
 #endif
 #define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
 #define AGC_MAX_R 4096         // straggler realisations per decode call
+#ifndef AGC_DEC_QT
+#define AGC_DEC_QT 16          // pack blocks per decode tile = consumer warps of the ring decoder
+#endif
+#ifndef AGC_DEC_GROUP_BITS
+#define AGC_DEC_GROUP_BITS 48  // cap on sum of b_i over a worker group: stage = QT * 64 * this bytes
+#endif
+#define AGC_DEC_MAX_STAGES 4
+#define AGC_DEC_RING_MAX_WORKERS 2048  // above this the per-worker tables no longer fit shared memory
 #define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
 #define AGC_STATIC_MAX_R 4096
 
@@ -83,6 +91,8 @@ struct AgcDecParams {
     int rows_per_bucket;
     float lr0;              // learning rate of the single realisation (R == 1)
     const float *lr;        // device, R learning rates (per-realisation mode with beta)
+    uint32_t *status = nullptr;  // AGC_STATUS_* bits are OR-ed into it (ring kernel), may be NULL
+    int stages = 0;              // ring depth of the ring kernel
 };
 
 struct agc_plan {
@@ -100,6 +110,10 @@ struct agc_plan {
     bool use_tma = false;
     int n_groups = 0, stage_rows = 0, stages = 0;
     size_t enc_smem = 0;
+    // decode ring
+    bool dec_ring = false;
+    int dec_stages = 0;
+    size_t dec_smem = 0;
     // device tables
     int32_t *d_row_ptr = nullptr, *d_col_idx = nullptr;
     float *d_a = nullptr, *d_w = nullptr;
@@ -122,4 +136,5 @@ struct agc_plan {
 int agc_launch_encode(agc_plan *plan, const float *G, long long ld, uint64_t round, void *codes,
                       float *scales, uint32_t *status, cudaStream_t stream);
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
-                      int R, const float *lr_host, float *ghat, float *beta, cudaStream_t stream);
+                      int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
+                      cudaStream_t stream);

@@ -7,6 +7,7 @@
 #include "agc_internal.h"
 
 int agc_encode_prepare(agc_plan *plan);
+int agc_decode_prepare(agc_plan *plan, int smem_optin);
 
 namespace {
 
@@ -214,6 +215,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_lr), sizeof(float) * AGC_MAX_R) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc) rc = agc_encode_prepare(pl);
+    if (!rc) rc = agc_decode_prepare(pl, smem_optin);
     if (rc) {
         free_device(pl);
         delete pl;
@@ -253,7 +255,7 @@ extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t
 
 extern "C" int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
                           const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
-                          float *beta_dev, void *cuda_stream)
+                          float *beta_dev, uint32_t *status_dev, void *cuda_stream)
 {
     if (!plan || !codes_dev || !scales_dev || !masks_dev) return AGC_ERR_ARG;
     if (R < 1 || (!ghat_dev && !beta_dev) || (beta_dev && !lr_host)) return AGC_ERR_ARG;
@@ -261,7 +263,7 @@ extern "C" int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *
     if ((reinterpret_cast<uintptr_t>(codes_dev) & 15) || (ghat_dev && (reinterpret_cast<uintptr_t>(ghat_dev) & 15)) ||
         (beta_dev && (reinterpret_cast<uintptr_t>(beta_dev) & 15)))
         return AGC_ERR_ALIGN;
-    return agc_launch_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host, ghat_dev, beta_dev,
+    return agc_launch_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host, ghat_dev, beta_dev, status_dev,
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -288,7 +290,8 @@ extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_
         return AGC_ERR_CUDA;
     int rc = agc_launch_encode(plan, plan->h_G, ld_dev, round, plan->h_codes, plan->h_scales, plan->h_status, st);
     if (rc) return rc;
-    rc = agc_launch_decode(plan, plan->h_codes, plan->h_scales, plan->h_mask, 1, nullptr, plan->h_ghat, nullptr, st);
+    rc = agc_launch_decode(plan, plan->h_codes, plan->h_scales, plan->h_mask, 1, nullptr, plan->h_ghat, nullptr,
+                           plan->h_status, st);
     if (rc) return rc;
     uint32_t status = 0;
     if (cudaMemcpyAsync(ghat_host, plan->h_ghat, sizeof(float) * plan->d, cudaMemcpyDeviceToHost, st) != cudaSuccess ||

@@ -43,7 +43,7 @@ class Session:
         """masks: (R, n) uint8 CUDA tensor."""
         assert masks.dtype == torch.uint8 and masks.is_cuda and masks.is_contiguous()
         R = masks.shape[0] if masks.dim() == 2 else 1
-        B.agc_decode(self.plan, self.codes, self.scales, masks, R, lr, ghat, beta, stream)
+        B.agc_decode(self.plan, self.codes, self.scales, masks, R, lr, ghat, beta, self.status, stream)
 
     def worker_words(self, i):
         lo = B.agc_worker_offset(self.plan, i) // 4
