@@ -202,15 +202,76 @@ struct __align__(16) AgcDecWorker {
     uint32_t pad;
 };
 
+// (a & b) | c in one logic instruction
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// One worker's contribution to the lane's 16 accumulators, read from the staged chunk.
+//   tl   warp * 64 + lane * 2 (even widths: byte offset of the lane's slice is tl * BITS)
+//   to   warp * 64 + (lane / 2) * 4 (odd widths: a pair of lanes shares BITS words)
+// The integer code c becomes the float 2^23 + c by OR-ing it into the mantissa of 2^23
+// (one byte permute for 8-bit codes); level = that - (2^23 + L) is exact.
 template <int BITS>
-__device__ __forceinline__ void ring_add_worker(const unsigned char *chunk, int warp, int lane,
+__device__ __forceinline__ void ring_add_worker(const unsigned char *chunk, uint32_t tl, uint32_t to, int lane,
                                                 const float (&ws_row)[4], float (&acc)[16])
 {
-    constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)((1 << (BITS >= 2 ? BITS - 1 : 1)) - 1)) : 2.0f;
+    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+    constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)(BITS >= 2 ? L : 1u)) : 2.0f;
+    constexpr int NACC = (16 * BITS + 31) / 32;
     float cstep_row[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
-    unpack_accumulate<BITS, false>(reinterpret_cast<const uint32_t *>(chunk) + warp * 16 * BITS, lane, cstep_row, acc);
+    uint32_t A[NACC + 1];
+    A[NACC] = 0u;
+    if constexpr (BITS % 2 == 0) {
+        constexpr int NW = BITS / 2;
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(chunk + tl * BITS);
+        if constexpr (NW == 4) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(src);
+            A[0] = v.x; A[1] = v.y; A[2] = v.z; A[3] = v.w;
+        } else if constexpr (NW == 2) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(src);
+            A[0] = v.x; A[1] = v.y;
+        } else {
+#pragma unroll
+            for (int t = 0; t < NW; ++t) A[t] = src[t];
+        }
+    } else {
+        constexpr int H = (BITS - 1) / 2;
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(chunk + to * BITS) + ((lane & 1) ? H : 0);
+        uint32_t W[H + 1];
+#pragma unroll
+        for (int t = 0; t <= H; ++t) W[t] = src[t];
+        if (lane & 1) {
+#pragma unroll
+            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
+            A[H] = W[H] >> 16;
+        } else {
+#pragma unroll
+            for (int t = 0; t <= H; ++t) A[t] = W[t];
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+        const int bitpos = t * BITS;
+        const int w = bitpos >> 5, sh = bitpos & 31;
+        float level;
+        if constexpr (BITS == 1) {
+            level = __uint_as_float(0xBF000000u ^ ((A[0] >> t) << 31));                     // code - 0.5
+        } else {
+            uint32_t x;
+            if constexpr (BITS == 8) x = __byte_perm(A[w], 0x4B000000u, 0x7540u | (uint32_t)(sh >> 3));
+            else if (sh + BITS <= 32) x = and_or(sh ? A[w] >> sh : A[w], MASK, 0x4B000000u);
+            else x = and_or(__funnelshift_r(A[w], A[w + 1], sh), MASK, 0x4B000000u);
+            level = __fsub_rn(__uint_as_float(x), 8388608.0f + (float)L);                   // code - L, exact
+        }
+        acc[t] = __fmaf_rn(cstep_row[t >> 2], level, acc[t]);
+    }
 }
 
 template <int RB, bool COLLAPSED>
@@ -313,23 +374,20 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     } else {
         // ---------------- consumers: warp w owns pack block q0 + w of every tile
         const bool vec = (P.d & 3) == 0;
+        const uint32_t tl = (uint32_t)warp * 64u + (uint32_t)lane * 2u;
+        const uint32_t to = (uint32_t)warp * 64u + (uint32_t)(lane >> 1) * 4u;
         int s = 0;
         uint32_t parity = 0;
         bool ok = true;
-        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+        // scales of the lane's worker (lane < workers of the group) for this warp's block of a
+        // tile; fetched one tile ahead so that their latency hides behind the current tile
+        auto fetch_scales = [&](long long T, int g, float (&sc)[4 / RB]) {
+#pragma unroll
+            for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
             const long long q = T * AGC_DEC_QT + warp;
-            const bool active = q < P.nblk;
-            float acc[16], b[16];
-#pragma unroll
-            for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
-            if (P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
-            for (int g = 0; ok && g < n_groups; ++g) {
+            if (T < ntile && g < n_groups && q < P.nblk) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
-                // the lane's worker of this group: its scale(s) for block q, fetched before the wait
-                float sc[4 / RB];
-#pragma unroll
-                for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
-                if (active && lane < nr) {
+                if (lane < nr) {
                     const float *srow = P.scales + s_wk[r0 + lane].scales_off;
 #pragma unroll
                     for (int bk = 0; bk < 4 / RB; ++bk) {
@@ -337,6 +395,25 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                         if (beta_idx < P.nb) sc[bk] = __ldg(srow + beta_idx);
                     }
                 }
+            }
+        };
+        float sc_next[4 / RB];
+        fetch_scales(blockIdx.x, 0, sc_next);
+        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+            const long long q = T * AGC_DEC_QT + warp;
+            const bool active = q < P.nblk;
+            float acc[16], b[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+            for (int g = 0; ok && g < n_groups; ++g) {
+                const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
+                float sc[4 / RB];
+#pragma unroll
+                for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = sc_next[bk];
+                if (g + 1 < n_groups) fetch_scales(T, g + 1, sc_next);
+                else fetch_scales(T + gridDim.x, 0, sc_next);
+                // parameters of the block: read early, used after the last group
+                if (g == n_groups - 1 && P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
                 ok = mbar_wait(&full[s], parity, flags);
                 if (!ok) break;
                 if (active) {
@@ -353,14 +430,14 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                         }
                         const unsigned char *chunk = stage + wk.soff;
                         switch (wk.bits) {
-                            case 1: ring_add_worker<1>(chunk, warp, lane, ws_row, acc); break;
-                            case 2: ring_add_worker<2>(chunk, warp, lane, ws_row, acc); break;
-                            case 3: ring_add_worker<3>(chunk, warp, lane, ws_row, acc); break;
-                            case 4: ring_add_worker<4>(chunk, warp, lane, ws_row, acc); break;
-                            case 5: ring_add_worker<5>(chunk, warp, lane, ws_row, acc); break;
-                            case 6: ring_add_worker<6>(chunk, warp, lane, ws_row, acc); break;
-                            case 7: ring_add_worker<7>(chunk, warp, lane, ws_row, acc); break;
-                            default: ring_add_worker<8>(chunk, warp, lane, ws_row, acc); break;
+                            case 1: ring_add_worker<1>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 2: ring_add_worker<2>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 3: ring_add_worker<3>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 4: ring_add_worker<4>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 5: ring_add_worker<5>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 6: ring_add_worker<6>(chunk, tl, to, lane, ws_row, acc); break;
+                            case 7: ring_add_worker<7>(chunk, tl, to, lane, ws_row, acc); break;
+                            default: ring_add_worker<8>(chunk, tl, to, lane, ws_row, acc); break;
                         }
                     }
                 }
@@ -369,6 +446,7 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 if (++s == stages) { s = 0; parity ^= 1u; }
             }
             if (ok && active) {
+                if (n_groups == 0 && P.beta) load16(P.beta, q, lane, P.d, vec, b);
                 if (COLLAPSED) {
 #pragma unroll
                     for (int t = 0; t < 16; ++t) b[t] = __fsub_rn(b[t], acc[t]);

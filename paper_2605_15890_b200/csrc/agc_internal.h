@@ -17,12 +17,12 @@
 #define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
 #define AGC_MAX_R 4096         // straggler realisations per decode call
 #ifndef AGC_DEC_QT
-#define AGC_DEC_QT 16          // pack blocks per decode tile = consumer warps of the ring decoder
+#define AGC_DEC_QT 31          // pack blocks per decode tile = consumer warps of the ring decoder (+1 producer = 8 per scheduler)
 #endif
 #ifndef AGC_DEC_GROUP_BITS
-#define AGC_DEC_GROUP_BITS 48  // cap on sum of b_i over a worker group: stage = QT * 64 * this bytes
+#define AGC_DEC_GROUP_BITS 32  // cap on sum of b_i over a worker group: stage = QT * 64 * this bytes
 #endif
-#define AGC_DEC_MAX_STAGES 4
+#define AGC_DEC_MAX_STAGES 8
 #define AGC_DEC_RING_MAX_WORKERS 2048  // above this the per-worker tables no longer fit shared memory
 #define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
 #define AGC_STATIC_MAX_R 4096

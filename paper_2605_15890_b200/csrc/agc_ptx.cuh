@@ -31,16 +31,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(20000u) : "memory");
     return ok != 0;
 }
-// Bounded wait: each try suspends the warp in hardware for up to the hinted 20 us; after
-// 2^20 failed tries (a second at the very least) it gives up, records it and lets the
-// caller unwind.
+// Bounded wait. A warp that finds the phase incomplete sleeps between tries (64 ns doubling
+// to 1 us) instead of spinning, so that it does not take issue slots from the warps still
+// working; after about 2^20 tries (a second at the least) it gives up, records it and lets
+// the caller unwind.
+#ifndef AGC_WAIT_SLEEP_NS
+#define AGC_WAIT_SLEEP_NS 64u
+#endif
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
+    uint32_t ns = AGC_WAIT_SLEEP_NS;
     for (uint32_t spin = 0; spin < (1u << 20); ++spin) {
+        __nanosleep(ns);
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (spin > 16) __nanosleep(1000);
+        if (ns < 1024u) ns <<= 1;
+        else if (*abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
