@@ -218,6 +218,7 @@ def main():
 
     import torch
     import paper_2605_15890_b200 as agc
+    from paper_2605_15890_b200 import sharding
     from paper_2605_15890_b200.session import Session
     from synth import configs as cfgs
 
@@ -234,8 +235,11 @@ def main():
     code, bits = build_code(agc, wl, bucket)
     rp, ci, a, w = code
     flags = agc.AGC_FLAG_ALLOW_1BIT if int(bits.min()) == 1 else 0
-    wl.seed += rank  # each rank its own coordinate range: different data, same shape
+    # weak scaling: the job is a gradient of world * nblk pack blocks, rank r holds blocks
+    # [r * nblk, (r + 1) * nblk) of it (its own data, same shape), no exchange on the data path
     ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, bits, bucket=bucket, seed=wl.seed, flags=flags, device=dev)
+    ses.set_first_block(sharding.first_block(world * ((wl.d + 511) // 512) * 512, rank, world))
+    wl.seed += 7919 * rank  # the synthetic values of this rank's range
     ld = (wl.d + 3) // 4 * 4
     G = cfgs.partials_torch(wl, dev, ld=ld)
     R = wl.realizations
@@ -281,10 +285,7 @@ def main():
     k2_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
     step_ms = k1_ms + k2_ms if flush is not None else evs[0][0].elapsed_time(evs[-1][2]) / args.steps
     status = int(ses.status.item())
-    if dist:
-        tt = torch.tensor([step_ms, k1_ms, k2_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        step_ms, k1_ms, k2_ms = (float(x) for x in tt.cpu())
+    step_ms, k1_ms, k2_ms = sharding.max_over_ranks([step_ms, k1_ms, k2_ms], device=dev)
     value = world * wl.d / (step_ms * 1e-3)
 
     # end to end through the host-buffer entry point (pinned host memory, copies timed)
@@ -302,10 +303,7 @@ def main():
         for t in range(args.e2e_steps):
             agc.agc_round_host(ses.plan, Gh, wl.d, t + 1, mh, gh)
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-        if dist:
-            tt = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_s = float(tt.item())
+        e2e_s = sharding.max_over_ranks([e2e_s], device=dev)[0]
         e2e = {"value": world * wl.d / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 4 * wl.k * wl.d + wl.n,
                "d2h_bytes_per_step": 4 * wl.d + 4, "ms_per_step": 1e3 * e2e_s, "steps": args.e2e_steps}
         del Gh, gh

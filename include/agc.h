@@ -103,6 +103,17 @@ size_t agc_scales_bytes(const agc_plan_t *plan);
 /* Byte offset of worker i's message inside the codes buffer (multiple of 64);
  * i = n gives agc_codes_bytes. Returns (size_t)-1 for a bad index. */
 size_t agc_worker_offset(const agc_plan_t *plan, int i);
+/*
+ * agc_plan_set_first_block - place the plan's coordinates inside a longer vector.
+ * The random draw of the stochastic rounding (Eq. rv_quant) is keyed by the position of
+ * a coordinate in the worker's message. A plan that covers coordinates
+ * [512 * first_block, 512 * first_block + d) of a longer gradient - one shard of it on
+ * one GPU - then draws exactly what a plan over the whole vector draws there, and since
+ * every bucket has its own norm, the shard's codes and scales are the corresponding
+ * slices of the whole vector's. Default 0. first_block >= 0, first_block + ceil(d/512)
+ * <= 2^26. Takes effect from the next agc_encode_quantize.
+ */
+int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block);
 /* 1 if the plan encodes with the TMA-staged kernel, 0 if with the direct-load kernel. */
 int agc_plan_uses_tma(const agc_plan_t *plan);
 

@@ -51,6 +51,8 @@ def _load():
         getattr(L, name).restype = C.c_size_t
     L.agc_worker_offset.argtypes = [vp, C.c_int]
     L.agc_worker_offset.restype = C.c_size_t
+    L.agc_plan_set_first_block.argtypes = [vp, C.c_int64]
+    L.agc_plan_set_first_block.restype = C.c_int
     L.agc_plan_uses_tma.argtypes = [vp]
     L.agc_plan_uses_tma.restype = C.c_int
     L.agc_encode_quantize.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, vp, vp]
@@ -146,6 +148,10 @@ def agc_scales_bytes(plan):
 
 def agc_worker_offset(plan, i):
     return _lib.agc_worker_offset(plan, i)
+
+
+def agc_plan_set_first_block(plan, first_block):
+    _check(_lib.agc_plan_set_first_block(plan, first_block))
 
 
 def agc_plan_uses_tma(plan):

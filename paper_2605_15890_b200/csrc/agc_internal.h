@@ -70,6 +70,7 @@ struct AgcEncParams {
     float *scales;
     uint32_t *status;
     long long d, ld, nblk, nb;
+    long long first_block;       // pack-block index of coordinate 0 in the random stream
     int n, k, n_groups, nnz;
     int stages, stage_rows;
     uint32_t round_lo, round_hi;
@@ -100,6 +101,7 @@ struct agc_plan {
     long long d = 0, nblk = 0, nb = 0;
     int bucket = 0;
     uint64_t seed = 0;
+    long long first_block = 0;
     uint32_t flags = 0;
     int device = 0, sm_count = 0;
     std::vector<int32_t> row_ptr, col_idx;

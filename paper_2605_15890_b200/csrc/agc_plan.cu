@@ -239,6 +239,12 @@ extern "C" size_t agc_worker_offset(const agc_plan_t *plan, int i)
     if (!plan || i < 0 || i > plan->n) return size_t(-1);
     return size_t(plan->word_off[i]) * 4;
 }
+extern "C" int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block)
+{
+    if (!plan || first_block < 0 || first_block + plan->nblk > (int64_t(1) << 26)) return AGC_ERR_ARG;
+    plan->first_block = first_block;
+    return AGC_OK;
+}
 extern "C" int agc_plan_uses_tma(const agc_plan_t *plan) { return plan && plan->use_tma ? 1 : 0; }
 
 extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,

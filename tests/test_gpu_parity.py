@@ -229,3 +229,119 @@ def test_host_buffer_round(agc, torch):
         og, _ = orp.decode(wl.d, wl.bits, 512, w, mask.numpy()[None], oc, osc)
         assert (ghat.numpy().view(np.uint32) == og[0].view(np.uint32)).all()
     ses.close()
+
+
+def test_shards_with_block_offsets_reproduce_the_whole_vector(agc, torch):
+    """The multi-GPU recipe on one GPU: two plans over pack-block-aligned halves, each told
+    its first block, give the corresponding slices of the whole vector's codes and scales."""
+    from paper_2605_15890_b200 import sharding
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(8)
+    n = k = 6
+    d = 512 * 9 + 77
+    B = 128
+    bits = np.array([2, 3, 4, 5, 7, 8], np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B)
+    G_host = rng.standard_normal((k, d)).astype(np.float32)
+    oc, osc, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 31, 2, G_host)
+    off = orp.worker_word_offsets(d, bits)
+    for rank in range(2):
+        lo, hi = sharding.coordinate_range(d, rank, 2)
+        ds = hi - lo
+        ses = Session(n, k, ds, rp, ci, a, w, p, bits, bucket=B, seed=31)
+        ses.set_first_block(sharding.first_block(d, rank, 2))
+        ld = (ds + 3) // 4 * 4
+        G = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+        G[:, :ds] = torch.from_numpy(np.ascontiguousarray(G_host[:, lo:hi]))
+        ses.encode(G, 2)
+        torch.cuda.synchronize()
+        codes, scales = ses.codes_host(), ses.scales_host()
+        nblk_s = (ds + 511) // 512
+        q0 = lo // 512
+        for i in range(n):
+            b = int(bits[i])
+            w_lo, w_hi = ses.worker_words(i)
+            assert w_hi - w_lo == nblk_s * 16 * b
+            want = oc[off[i] + q0 * 16 * b: off[i] + (q0 + nblk_s) * 16 * b]
+            assert (codes[w_lo:w_hi] == want).all()
+        nb_s = scales.shape[1]
+        assert (scales.view(np.uint32) == osc[:, lo // B: lo // B + nb_s].view(np.uint32)).all()
+        ses.close()
+
+
+def test_config5_shape_one_bit_workers_and_64_realisations(agc, torch):
+    """cfg5's structure at a size the oracle finishes: n=k=100, s=5, Student-t(3) values,
+    bits 1..8, 64 realisations decoded per encode with the update fused."""
+    wl = cfgs.config5(d=40_000 + 13)
+    code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
+    G = cfgs.partials_numpy(wl, 0)
+    masks = cfgs.straggler_masks(wl, rounds=1)[0]
+    rng = np.random.default_rng(1)
+    lr = rng.uniform(1e-4, 1e-3, wl.realizations).astype(np.float32)
+    beta0 = rng.standard_normal(wl.d).astype(np.float32)
+    out, ref = run_both(agc, torch, G, code, wl.p, wl.bits, 512, wl.seed, 0, masks, lr=lr, beta0=beta0)
+    assert_exact(out, ref)
+    assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
+    rel = np.abs(out["beta_fused"] - ref["beta"]).max() / np.abs(ref["beta"]).max()
+    assert rel <= 1e-5
+
+
+def test_config3_full_size_sampled_blocks(agc, torch):
+    """The benchmark's own configuration (d = 25,557,032, bits from the allocator, bucket 512,
+    the launch shape bench.py times): pack blocks sampled across the vector - first, last
+    (ragged), segment boundaries, random ones - are recomputed one by one by the oracle from
+    the same inputs and compared bit for bit: codes, scales, decode and fused update."""
+    from paper_2605_15890_b200.session import Session
+    wl = cfgs.config3()
+    B = 512
+    bits, _ = od.bit_allocate_low_complexity(wl.p, wl.z_tot, B, b_max=8)
+    bits = np.asarray(bits, np.uint8)
+    rp, ci, a, w = _codes.cyclic_code(wl.p, bits, wl.k, wl.s, B)
+    ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, bits, bucket=B, seed=wl.seed)
+    assert ses.uses_tma
+    ld = (wl.d + 3) // 4 * 4
+    G = cfgs.partials_torch(wl, "cuda:0", ld=ld)
+    mask = cfgs.straggler_masks(wl, rounds=1)[0]
+    m_dev = torch.from_numpy(mask).cuda()
+    ghat = torch.empty((1, wl.d), dtype=torch.float32, device="cuda")
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(77)
+    beta0 = torch.empty(wl.d, dtype=torch.float32, device="cuda").normal_(generator=gen)
+    beta = beta0.clone()
+    lr = np.array([0.05], np.float32)
+    rnd = 11
+    ses.encode(G, rnd)
+    ses.decode(m_dev, lr=lr, ghat=ghat, beta=beta)
+    torch.cuda.synchronize()
+    assert int(ses.status.item()) == 0
+    nblk = (wl.d + 511) // 512
+    starts, _, _ = cfgs.segment_table(wl)
+    rng = np.random.default_rng(3)
+    sample = {0, 1, nblk - 2, nblk - 1} | {int(s_) // 512 for s_ in starts[1:40]} | \
+        {int(x) for x in rng.integers(0, nblk, 200)}
+    off = orp.worker_word_offsets(wl.d, bits)
+    codes = ses.codes
+    for q in sorted(sample):
+        m0, m1 = q * 512, min((q + 1) * 512, wl.d)
+        blk = np.zeros((wl.k, 512), np.float32)
+        blk[:, :m1 - m0] = G[:, m0:m1].cpu().numpy()
+        oc, osc, st, _ = orp.encode_block(rp, ci, a, bits, B, wl.seed, rnd, q, blk)
+        assert st == 0
+        wb = 0
+        for i in range(wl.n):
+            b = int(bits[i])
+            lo = int(off[i]) + q * 16 * b
+            got = codes[lo:lo + 16 * b].cpu().numpy().view(np.uint32)
+            assert (got == oc[wb:wb + 16 * b]).all(), (q, i)
+            wb += 16 * b
+        got_s = ses.scales.view(wl.n, -1)[:, q].cpu().numpy()
+        assert (got_s.view(np.uint32) == osc[:, 0].view(np.uint32)).all(), q
+        og = orp.decode_block(bits, B, w, mask[0], oc, osc)
+        gg = ghat[0, m0:m1].cpu().numpy()
+        assert (gg.view(np.uint32) == og[:m1 - m0].view(np.uint32)).all(), q
+        ob = np.float32(beta0[m0:m1].cpu().numpy())
+        want_b = (ob.astype(np.float64) - np.float64(lr[0]) * og[:m1 - m0].astype(np.float64))
+        # fused update is one fp32 fma: compare against the correctly rounded value
+        assert (beta[m0:m1].cpu().numpy() == want_b.astype(np.float32)).all(), q
+    ses.close()

@@ -1,0 +1,102 @@
+"""Two CPU ranks (gloo): the sharding recipe of the multi-GPU path. Each rank takes its
+pack-block-aligned coordinate range, encodes it on its own with the global block indices
+in the random stream, and the gathered pieces must equal the encoding of the whole vector;
+step times are reduced with a maximum over ranks. No GPU is involved: the per-shard encode
+is done by the CPU oracle, the range / reduction logic is the product's."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import roundpath as orp
+from paper_2605_15890_b200 import sharding
+from tests import _codes
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _problem():
+    rng = np.random.default_rng(5)
+    n = k = 4
+    d = 512 * 7 + 100            # 8 pack blocks, ragged tail
+    bits = np.array([2, 3, 5, 8], np.uint8)
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    code = _codes.cyclic_code(p, bits, k, 2, 256)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    return n, k, d, bits, code, G
+
+
+def _rank_main(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        n, k, d, bits, (rp, ci, a, w), G = _problem()
+        B, seed, rnd = 256, 9, 4
+        lo, hi = sharding.coordinate_range(d, rank, world)
+        q0 = sharding.first_block(d, rank, world)
+        pieces = []
+        for q in range(q0, q0 + (hi - lo + 511) // 512):
+            blk = np.zeros((k, 512), np.float32)
+            m0, m1 = q * 512, min((q + 1) * 512, d)
+            blk[:, :m1 - m0] = G[:, m0:m1]
+            c, s, st, _ = orp.encode_block(rp, ci, a, bits, B, seed, rnd, q, blk)
+            assert st == 0
+            pieces.append((q, c, s))
+        gathered = [None] * world
+        dist.all_gather_object(gathered, (lo, hi, pieces))
+        ms = sharding.max_over_ranks([10.0 + rank, 5.0 - rank])
+        if rank == 0:
+            whole_c, whole_s, st, _ = orp.encode_quantize(rp, ci, a, bits, B, seed, rnd, G)
+            off = orp.worker_word_offsets(d, bits)
+            covered = np.zeros(d, bool)
+            for glo, ghi, gp in gathered:
+                assert not covered[glo:ghi].any()
+                covered[glo:ghi] = True
+                for q, c, s in gp:
+                    wb = 0
+                    for i in range(n):
+                        b = int(bits[i])
+                        got = c[wb:wb + 16 * b]
+                        want = whole_c[off[i] + q * 16 * b: off[i] + (q + 1) * 16 * b]
+                        assert (got == want).all(), (q, i)
+                        wb += 16 * b
+                        for bk in range(512 // B):
+                            beta = q * (512 // B) + bk
+                            if beta < whole_s.shape[1]:
+                                assert s[i, bk].view(np.uint32) == whole_s[i, beta].view(np.uint32)
+            assert covered.all()
+            assert ms == [10.0 + world - 1, 5.0]
+            with open(os.path.join(out_dir, "ok"), "w") as fh:
+                fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_whole_encoding(tmp_path):
+    world = 2
+    mp.spawn(_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    assert (tmp_path / "ok").exists()
+
+
+@pytest.mark.parametrize("d,world", [(0, 3), (1, 2), (511, 2), (512, 2), (513, 4), (25_557_032, 8), (10**8, 3)])
+def test_coordinate_ranges_tile_the_vector(d, world):
+    prev = 0
+    for r in range(world):
+        lo, hi = sharding.coordinate_range(d, r, world)
+        assert lo == prev and lo <= hi <= d
+        assert lo % 512 == 0 or lo == d
+        assert sharding.first_block(d, r, world) * 512 == lo or lo == d
+        prev = hi
+    assert prev == d
+    sizes = [sharding.coordinate_range(d, r, world) for r in range(world)]
+    blocks = [(hi - lo + 511) // 512 for lo, hi in sizes]
+    assert max(blocks) - min(blocks) <= 1
