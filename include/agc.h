@@ -263,6 +263,16 @@ int agc_code_build(int n, int k, const double *p, const uint8_t *bits, double ph
                    const int32_t *sup_col_idx, int32_t nnz_cap, int32_t *row_ptr_out,
                    int32_t *col_out, float *a_out, float *w_out, double *Y_out);
 
+/*
+ * agc_selftest_division - diagnostic. The encoder forms the reciprocal scale L_i 2^15 / S
+ * of Eq. quant_def's normalisation with its own branch-free division; this call compares
+ * it on the current device with the IEEE-754 correctly rounded quotient for every
+ * numerator and every float S the encoder can meet (about 8.5e9 pairs, a few seconds)
+ * and writes the number of differing results (expected 0) to *mismatches_out (host).
+ * Synchronous; allocates 8 bytes of device memory for the duration of the call.
+ */
+int agc_selftest_division(unsigned long long *mismatches_out);
+
 /* Human-readable text for an AGC_ERR_* code (static storage). */
 const char *agc_strerror(int code);
 /* Library version: major*10000 + minor*100 + patch. */

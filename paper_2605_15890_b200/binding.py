@@ -71,6 +71,8 @@ def _load():
     L.agc_code_build.argtypes = [C.c_int, C.c_int, f64p, u8p, C.c_double, C.c_double, C.c_int, i32p,
                                  i32p, C.c_int32, i32p, i32p, f32p, f32p, f64p]
     L.agc_code_build.restype = C.c_int
+    L.agc_selftest_division.argtypes = [C.POINTER(C.c_ulonglong)]
+    L.agc_selftest_division.restype = C.c_int
     L.agc_strerror.argtypes = [C.c_int]
     L.agc_strerror.restype = C.c_char_p
     L.agc_version.argtypes = []
@@ -196,6 +198,14 @@ def agc_round_host(plan, G_host, ld_host, rnd, mask_host, ghat_host, stream=None
     _check(_lib.agc_round_host(plan, addr(G_host), ld_host, rnd, addr(mask_host), addr(ghat_host),
                                C.byref(st), _stream(stream)))
     return st.value
+
+
+def agc_selftest_division():
+    """Number of (numerator, scale) pairs for which the encoder's division differs from the
+    correctly rounded quotient (expected 0)."""
+    bad = C.c_ulonglong(0)
+    _check(_lib.agc_selftest_division(C.byref(bad)))
+    return bad.value
 
 
 def _alloc(fn, p, z_tot, b_min, b_max, phi_dim, eta):

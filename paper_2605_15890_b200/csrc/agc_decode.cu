@@ -186,6 +186,9 @@ __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *
     weff[i] = s;
 }
 
+#ifndef AGC_DEC_PREFETCH
+#define AGC_DEC_PREFETCH 1
+#endif
 // ------------------------------------------------------------------ ring kernel
 // Persistent CTAs. A tile is AGC_DEC_QT consecutive pack blocks of one group of received
 // workers: the producer warp brings each worker's chunk (its words of those blocks are
@@ -199,7 +202,7 @@ struct __align__(16) AgcDecWorker {
     float weight;          // w_i, or w_i * (sum_r lr_r I_ri) in the collapsed mode
     uint32_t soff;         // byte offset of the worker's chunk inside a stage
     uint32_t bits;
-    uint32_t pad;
+    uint32_t run;          // at the first worker of a run of equal widths inside a group: its length
 };
 
 // (a & b) | c in one logic instruction
@@ -210,13 +213,33 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
     return d;
 }
 
-// One worker's contribution to the lane's 16 accumulators, read from the staged chunk.
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// One worker's contribution to the lane's 16 accumulators, read from the staged chunk
+// (chunk: its 32-bit shared-memory address).
 //   tl   warp * 64 + lane * 2 (even widths: byte offset of the lane's slice is tl * BITS)
 //   to   warp * 64 + (lane / 2) * 4 (odd widths: a pair of lanes shares BITS words)
 // The integer code c becomes the float 2^23 + c by OR-ing it into the mantissa of 2^23
 // (one byte permute for 8-bit codes); level = that - (2^23 + L) is exact.
 template <int BITS>
-__device__ __forceinline__ void ring_add_worker(const unsigned char *chunk, uint32_t tl, uint32_t to, int lane,
+__device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uint32_t to, int lane,
                                                 const float (&ws_row)[4], float (&acc)[16])
 {
     constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
@@ -230,23 +253,23 @@ __device__ __forceinline__ void ring_add_worker(const unsigned char *chunk, uint
     A[NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
         constexpr int NW = BITS / 2;
-        const uint32_t *src = reinterpret_cast<const uint32_t *>(chunk + tl * BITS);
+        const uint32_t src = chunk + tl * BITS;
         if constexpr (NW == 4) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(src);
+            const uint4 v = lds128(src);
             A[0] = v.x; A[1] = v.y; A[2] = v.z; A[3] = v.w;
         } else if constexpr (NW == 2) {
-            const uint2 v = *reinterpret_cast<const uint2 *>(src);
+            const uint2 v = lds64(src);
             A[0] = v.x; A[1] = v.y;
         } else {
 #pragma unroll
-            for (int t = 0; t < NW; ++t) A[t] = src[t];
+            for (int t = 0; t < NW; ++t) A[t] = lds32(src + 4 * t);
         }
     } else {
         constexpr int H = (BITS - 1) / 2;
-        const uint32_t *src = reinterpret_cast<const uint32_t *>(chunk + to * BITS) + ((lane & 1) ? H : 0);
+        const uint32_t src = chunk + to * BITS + ((lane & 1) ? 4 * H : 0);
         uint32_t W[H + 1];
 #pragma unroll
-        for (int t = 0; t <= H; ++t) W[t] = src[t];
+        for (int t = 0; t <= H; ++t) W[t] = lds32(src + 4 * t);
         if (lane & 1) {
 #pragma unroll
             for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
@@ -299,7 +322,7 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
         asm volatile("fence.proxy.async;" ::: "memory");
         // compact list of the workers that contribute, cut into groups of at most 32 workers
         // and AGC_DEC_GROUP_BITS bits per coordinate
-        int nrecv = 0, ng = 0, in_grp = 0;
+        int nrecv = 0, ng = 0, in_grp = 0, run_head = 0;
         uint32_t grp_bits = 0, soff = 0;
         s_grp_ptr[0] = 0;
         for (int i = 0; i < P.n; ++i) {
@@ -317,13 +340,18 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 s_grp_ptr[++ng] = nrecv;
                 in_grp = 0; grp_bits = 0; soff = 0;
             }
+            if (in_grp && s_wk[run_head].bits == b) {
+                s_wk[run_head].run += 1;
+            } else {
+                run_head = nrecv;
+            }
             AgcDecWorker wk;
             wk.word_off = P.word_off[i];
             wk.scales_off = (long long)i * P.nb;
             wk.weight = wgt;
             wk.soff = soff;
             wk.bits = b;
-            wk.pad = 0;
+            wk.run = 1;
             s_wk[nrecv++] = wk;
             soff += AGC_DEC_QT * 64u * b;
             grp_bits += b;
@@ -347,10 +375,11 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
             const uint32_t nq = (uint32_t)(P.nblk - q0 < AGC_DEC_QT ? P.nblk - q0 : AGC_DEC_QT);
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
-                uint32_t bytes = 0, soff = 0;
+                uint32_t bytes = 0, soff = 0, wbits = 0;
                 const unsigned char *src = nullptr;
                 if (lane < nr) {
                     const AgcDecWorker wk = s_wk[r0 + lane];
+                    wbits = wk.bits;
                     bytes = nq * 64u * wk.bits;
                     soff = wk.soff;
                     src = reinterpret_cast<const unsigned char *>(P.codes + wk.word_off + q0 * 16 * wk.bits);
@@ -358,11 +387,22 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 uint32_t total = bytes;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
-                ok = mbar_wait(&empty[s], parity, flags);
+                ok = mbar_wait<AGC_PRODUCER_SLEEP_NS>(&empty[s], parity, flags);
                 if (!ok) break;
                 if (lane == 0) mbar_arrive_expect_tx(&full[s], total);
                 __syncwarp();
-                if (lane < nr) bulk_load_1d(smem + (size_t)s * stage_bytes + soff, src, bytes, &full[s]);
+                if (lane < nr) {
+                    bulk_load_1d(smem + (size_t)s * stage_bytes + soff, src, bytes, &full[s]);
+#if AGC_DEC_PREFETCH
+                    // the same workers' chunks of this CTA's next tile row: on their way to L2 a
+                    // whole tile row ahead, so that the ring refills at L2 latency, not HBM latency
+                    const long long qn = q0 + (long long)gridDim.x * AGC_DEC_QT;
+                    if (qn < P.nblk) {
+                        const uint32_t nqn = (uint32_t)(P.nblk - qn < AGC_DEC_QT ? P.nblk - qn : AGC_DEC_QT);
+                        bulk_prefetch_l2(src + (size_t)gridDim.x * AGC_DEC_QT * 64u * wbits, nqn * 64u * wbits);
+                    }
+#endif
+                }
                 ++issued;
                 if (++s == stages) { s = 0; parity ^= 1u; }
             }
@@ -417,28 +457,34 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 ok = mbar_wait(&full[s], parity, flags);
                 if (!ok) break;
                 if (active) {
-                    const unsigned char *stage = smem + (size_t)s * stage_bytes;
-                    for (int r = 0; r < nr; ++r) {
-                        const AgcDecWorker wk = s_wk[r0 + r];
-                        float ws_row[4];
-#pragma unroll
-                        for (int bk = 0; bk < 4 / RB; ++bk) {
-                            const float S = __shfl_sync(0xffffffffu, sc[bk], r);
-                            const float ws = __fmul_rn(wk.weight, S);
-#pragma unroll
-                            for (int cc = 0; cc < RB; ++cc) ws_row[bk * RB + cc] = ws;
+                    const uint32_t stage = smem_addr(smem) + (uint32_t)s * stage_bytes;
+                    // runs of workers of equal width: one dispatch per run
+                    for (int r = 0; r < nr;) {
+                        const int run = (int)s_wk[r0 + r].run;
+                        const uint32_t bits = s_wk[r0 + r].bits;
+#define AGC_DEC_RUN(B)                                                                          \
+    for (int j = 0; j < run; ++j) {                                                             \
+        const float weight = s_wk[r0 + r + j].weight;                                           \
+        const uint32_t chunk = stage + s_wk[r0 + r + j].soff;                                   \
+        float ws_row[4];                                                                        \
+        _Pragma("unroll") for (int bk = 0; bk < 4 / RB; ++bk) {                                 \
+            const float ws = __fmul_rn(weight, __shfl_sync(0xffffffffu, sc[bk], r + j));        \
+            _Pragma("unroll") for (int cc = 0; cc < RB; ++cc) ws_row[bk * RB + cc] = ws;        \
+        }                                                                                       \
+        ring_add_worker<B>(chunk, tl, to, lane, ws_row, acc);                                   \
+    }
+                        switch (bits) {
+                            case 1: AGC_DEC_RUN(1) break;
+                            case 2: AGC_DEC_RUN(2) break;
+                            case 3: AGC_DEC_RUN(3) break;
+                            case 4: AGC_DEC_RUN(4) break;
+                            case 5: AGC_DEC_RUN(5) break;
+                            case 6: AGC_DEC_RUN(6) break;
+                            case 7: AGC_DEC_RUN(7) break;
+                            default: AGC_DEC_RUN(8) break;
                         }
-                        const unsigned char *chunk = stage + wk.soff;
-                        switch (wk.bits) {
-                            case 1: ring_add_worker<1>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 2: ring_add_worker<2>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 3: ring_add_worker<3>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 4: ring_add_worker<4>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 5: ring_add_worker<5>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 6: ring_add_worker<6>(chunk, tl, to, lane, ws_row, acc); break;
-                            case 7: ring_add_worker<7>(chunk, tl, to, lane, ws_row, acc); break;
-                            default: ring_add_worker<8>(chunk, tl, to, lane, ws_row, acc); break;
-                        }
+#undef AGC_DEC_RUN
+                        r += run;
                     }
                 }
                 __syncwarp();

@@ -15,6 +15,9 @@
 #define AGC_ENC_CONSUMER_WARPS 23  // + 1 producer warp = 6 warps per scheduler at 80 registers
 #endif
 #define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
+#ifndef AGC_PRODUCER_SLEEP_NS
+#define AGC_PRODUCER_SLEEP_NS 32u  // cap of the producer warps' sleep between tries of a wait
+#endif
 #define AGC_MAX_R 4096         // straggler realisations per decode call
 #ifndef AGC_DEC_QT
 #define AGC_DEC_QT 31          // pack blocks per decode tile = consumer warps of the ring decoder (+1 producer = 8 per scheduler)
@@ -35,7 +38,8 @@ struct __align__(16) AgcWorkerDesc {
     uint16_t ne;           // entries in that row
     uint8_t bits;
     uint8_t pad;
-    uint32_t pad2[2];
+    float enc_scale;       // L_i * 2^15 (b_i >= 2) or 2^14 (b_i = 1)
+    uint32_t pad2;
 };
 struct __align__(8) AgcEntryDesc {
     float a;              // coefficient a_ij

@@ -169,7 +169,8 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     for (int i = 0; i < n_workers; ++i) {
         wdesc[i].word_off = pl->word_off[i];
         wdesc[i].scales_off = (long long)i * pl->nb;
-        wdesc[i].pad2[0] = wdesc[i].pad2[1] = 0;
+        wdesc[i].enc_scale = bits[i] >= 2 ? float(((1 << (bits[i] - 1)) - 1) << AGC_FRAC_BITS) : 16384.0f;
+        wdesc[i].pad2 = 0;
         wdesc[i].e0 = uint32_t(row_ptr[i]);
         wdesc[i].ne = uint16_t(std::min(row_ptr[i + 1] - row_ptr[i], 65535));
         wdesc[i].bits = bits[i];

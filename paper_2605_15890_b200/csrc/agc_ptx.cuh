@@ -31,21 +31,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(20000u) : "memory");
     return ok != 0;
 }
-// Bounded wait. A warp that finds the phase incomplete sleeps between tries (64 ns doubling
-// to 1 us) instead of spinning, so that it does not take issue slots from the warps still
-// working; after about 2^20 tries (a second at the least) it gives up, records it and lets
-// the caller unwind.
-#ifndef AGC_WAIT_SLEEP_NS
-#define AGC_WAIT_SLEEP_NS 64u
-#endif
+// Bounded wait. A warp that finds the phase incomplete sleeps between tries (32 ns doubling
+// up to MAX_SLEEP_NS) instead of spinning, so that it does not take issue slots from the
+// warps still working; a producer warp, whose wake-up delay adds to the refill latency of a
+// ring stage, uses a short cap. After 2^22 tries (a quarter of a second at the least with
+// the hardware's own suspension of each try) it gives up, records it and lets the caller
+// unwind.
+template <uint32_t MAX_SLEEP_NS = 512u>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    uint32_t ns = AGC_WAIT_SLEEP_NS;
-    for (uint32_t spin = 0; spin < (1u << 20); ++spin) {
+    uint32_t ns = 32u;
+    for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
         __nanosleep(ns);
         if (mbar_try_wait(bar, parity)) return true;
-        if (ns < 1024u) ns <<= 1;
+        if (ns < MAX_SLEEP_NS) ns <<= 1;
         else if (*abort_flag) return false;
     }
     *abort_flag = 1;
@@ -63,6 +63,13 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// Ask for a range of global memory (16-byte aligned, a multiple of 16 bytes) to be brought
+// into L2; no completion is signalled and nothing is written.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 
 }  // namespace

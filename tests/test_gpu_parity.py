@@ -345,3 +345,9 @@ def test_config3_full_size_sampled_blocks(agc, torch):
         # fused update is one fp32 fma: compare against the correctly rounded value
         assert (beta[m0:m1].cpu().numpy() == want_b.astype(np.float32)).all(), q
     ses.close()
+
+
+def test_encoder_division_is_correctly_rounded_everywhere(agc):
+    """The encoder's branch-free L 2^15 / S against the IEEE quotient for all eight
+    numerators and every float S in [2^-63, 2^64)."""
+    assert agc.agc_selftest_division() == 0
