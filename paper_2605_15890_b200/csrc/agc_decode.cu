@@ -308,6 +308,9 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     volatile int *flags = reinterpret_cast<volatile int *>(empty + AGC_DEC_MAX_STAGES);  // abort x2, n_groups
     AgcDecWorker *s_wk = reinterpret_cast<AgcDecWorker *>(empty + AGC_DEC_MAX_STAGES + 2);
     int32_t *s_grp_ptr = reinterpret_cast<int32_t *>(s_wk + P.n);
+    float *s_raw_w = reinterpret_cast<float *>(s_grp_ptr + P.n + 1);
+    uint8_t *s_raw_b = reinterpret_cast<uint8_t *>(s_raw_w + P.n);
+    uint8_t *s_raw_allb = s_raw_b + P.n;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -320,22 +323,37 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
         flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async;" ::: "memory");
+    }
+    // every thread fetches the inputs of some workers (weight, width; width 0 = contributes
+    // nothing), then one thread compacts them: the serial part touches shared memory only
+    for (int i = threadIdx.x; i < P.n; i += blockDim.x) {
+        float wgt = 0.0f;
+        bool used;
+        if (COLLAPSED) {
+            const float we = P.weff[i];
+            used = we != 0.0f;
+            if (used) wgt = __fmul_rn(P.w[i], we);
+        } else {
+            used = P.masks[i] != 0;
+            if (used) wgt = P.w[i];
+        }
+        s_raw_w[i] = wgt;
+        s_raw_b[i] = used ? P.bits[i] : (uint8_t)0;
+        s_raw_allb[i] = P.bits[i];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
         // compact list of the workers that contribute, cut into groups of at most 32 workers
         // and AGC_DEC_GROUP_BITS bits per coordinate
         int nrecv = 0, ng = 0, in_grp = 0, run_head = 0;
         uint32_t grp_bits = 0, soff = 0;
+        long long word_off = 0;
         s_grp_ptr[0] = 0;
         for (int i = 0; i < P.n; ++i) {
-            float wgt;
-            if (COLLAPSED) {
-                const float we = P.weff[i];
-                if (we == 0.0f) continue;
-                wgt = __fmul_rn(P.w[i], we);
-            } else {
-                if (!P.masks[i]) continue;
-                wgt = P.w[i];
-            }
-            const uint32_t b = P.bits[i];
+            const uint32_t b = s_raw_b[i];
+            const long long my_off = word_off;
+            word_off += P.nblk * 16 * (long long)s_raw_allb[i];
+            if (b == 0) continue;
             if (in_grp == 32 || grp_bits + b > AGC_DEC_GROUP_BITS) {
                 s_grp_ptr[++ng] = nrecv;
                 in_grp = 0; grp_bits = 0; soff = 0;
@@ -346,9 +364,9 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 run_head = nrecv;
             }
             AgcDecWorker wk;
-            wk.word_off = P.word_off[i];
+            wk.word_off = my_off;
             wk.scales_off = (long long)i * P.nb;
-            wk.weight = wgt;
+            wk.weight = s_raw_w[i];
             wk.soff = soff;
             wk.bits = b;
             wk.run = 1;
@@ -595,7 +613,7 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
     if ((plan->flags & AGC_FLAG_FORCE_DIRECT) || plan->n > AGC_DEC_RING_MAX_WORKERS) return AGC_OK;
     const size_t stage_bytes = size_t(AGC_DEC_QT) * 64 * AGC_DEC_GROUP_BITS;
     const size_t tail = (2 * AGC_DEC_MAX_STAGES + 2) * sizeof(uint64_t) + sizeof(AgcDecWorker) * size_t(plan->n) +
-                        sizeof(int32_t) * (size_t(plan->n) + 1) + 16;
+                        sizeof(int32_t) * (size_t(plan->n) + 1) + 6 * size_t(plan->n) + 16;
     if (size_t(smem_optin) < tail + 2 * stage_bytes) return AGC_OK;
     long long stages = (long long)((size_t(smem_optin) - tail) / stage_bytes);
     if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
