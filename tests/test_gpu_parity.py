@@ -351,3 +351,44 @@ def test_encoder_division_is_correctly_rounded_everywhere(agc):
     """The encoder's branch-free L 2^15 / S against the IEEE quotient for all eight
     numerators and every float S in [2^-63, 2^64)."""
     assert agc.agc_selftest_division() == 0
+
+
+def test_config4_least_squares_descent_in_lock_step(agc, torch):
+    """cfg4: least squares with 2^20 rows x 4,096 features split into 64 partitions, n = 64
+    workers, s = 2, bits 2..6; 500 rounds of gradient descent with the fused decode + update.
+    The partial gradients X_j^T (X_j w - y_j) come from torch (harness only). Every round the
+    oracle repeats encode, decode and update from the SAME partials and parameters: the
+    parameters after the round must agree bit for bit, so the two loss curves coincide; the
+    loss itself must fall from its start towards the noise floor."""
+    from paper_2605_15890_b200.session import Session
+    wl = cfgs.config4()
+    rows = wl.extra["rows"]
+    free, _ = torch.cuda.mem_get_info()
+    while rows * wl.d * 4 * 1.3 > free and rows > 65536:
+        rows //= 2                      # smaller boxes: fewer rows, same coding path
+    X, y, _ = cfgs.least_squares_problem(wl, "cuda:0", rows=rows)
+    B = 512
+    rp, ci, a, w = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, B)
+    ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, wl.bits, bucket=B, seed=wl.seed)
+    masks = cfgs.straggler_masks(wl)
+    m_dev = torch.from_numpy(masks).cuda()
+    lr = np.array([0.5 / rows], np.float32)
+    beta = torch.zeros(wl.d, dtype=torch.float32, device="cuda")
+    Xb = X.view(wl.k, rows // wl.k, wl.d)
+    losses = []
+    for t in range(wl.rounds):
+        r = X @ beta - y
+        losses.append(0.5 * float((r.double() ** 2).sum()))
+        G = torch.bmm(Xb.transpose(1, 2), r.view(wl.k, rows // wl.k, 1)).squeeze(2).contiguous()
+        beta_before = beta.cpu().numpy()
+        ses.encode(G, t)
+        ses.decode(m_dev[t], lr=lr, beta=beta)
+        G_host = G.cpu().numpy()
+        oc, osc, st, _ = orp.encode_quantize(rp, ci, a, wl.bits, B, wl.seed, t, G_host)
+        _, ob = orp.decode(wl.d, wl.bits, B, w, masks[t], oc, osc, lr=lr, beta=beta_before, want_ghat=False)
+        got = beta.cpu().numpy()
+        assert (got.view(np.uint32) == ob.view(np.uint32)).all(), f"round {t}"
+    assert int(ses.status.item()) == 0
+    ses.close()
+    assert losses[-1] < 0.05 * losses[0]
+    assert min(losses) == min(losses[-50:]) or losses[-1] < 1.5 * min(losses)
