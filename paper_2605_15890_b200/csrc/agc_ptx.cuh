@@ -37,10 +37,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // ring stage, uses a short cap. After 2^22 tries (a quarter of a second at the least with
 // the hardware's own suspension of each try) it gives up, records it and lets the caller
 // unwind.
-template <uint32_t MAX_SLEEP_NS = 512u>
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+template <uint32_t MAX_SLEEP_NS>
+__device__ __forceinline__ bool mbar_wait_loop(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     uint32_t ns = 32u;
     for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
         __nanosleep(ns);
@@ -50,6 +49,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     }
     *abort_flag = 1;
     return false;
+}
+template <uint32_t MAX_SLEEP_NS>
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    return mbar_wait_loop<MAX_SLEEP_NS>(bar, parity, abort_flag);
+}
+// OUT_OF_LINE keeps the retry loop out of the caller's instruction stream (measured: better
+// for the decoder's consumers, worse for the encoder's).
+template <uint32_t MAX_SLEEP_NS = 512u, bool OUT_OF_LINE = true>
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if constexpr (OUT_OF_LINE) return mbar_wait_slow<MAX_SLEEP_NS>(bar, parity, abort_flag);
+    else return mbar_wait_loop<MAX_SLEEP_NS>(bar, parity, abort_flag);
 }
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar)
 {
