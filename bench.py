@@ -29,7 +29,7 @@ UNIT = "coords/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the encode kernel, from the ncu
 # capture summarised under profiles/ (bytes per coordinate of the captured case, scaled to d).
-NCU_TRAFFIC_BYTES_PER_COORD = {}
+NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 142.28}   # profiles/k1_encode_staged_cfg3_d4M.md
 
 
 def workload(name):
