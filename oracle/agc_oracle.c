@@ -347,3 +347,34 @@ void agc_oracle_dequantize_worker(int64_t d, int b, int B, const uint32_t *codes
         out[m] = (scales_i[m / B] * dec_step(b)) * level;
     }
 }
+
+/*
+ * Adam step driven by the two-track estimates of Sec. V-E: the first moment follows g_w
+ * (the unbiased decode with w), the second moment follows g_v (the variance-reduced
+ * decode with v* of Eq. twodec); the step itself is Adam as published (Kingma & Ba, 2015,
+ * Algorithm 1). fp32, one IEEE operation per line:
+ *   m    <- (1-b1) * g_w   + b1 * m
+ *   u    <- (1-b2) * g_v^2 + b2 * u
+ *   beta <- beta - lr * (m * ibc1) / (sqrt(u * ibc2) + eps)
+ * c1 = 1 - b1, c2 = 1 - b2, ibc1 = 1 / (1 - b1^t), ibc2 = 1 / (1 - b2^t) (the bias
+ * corrections of step t): formed by the caller in double precision and rounded to fp32.
+ */
+void agc_oracle_adam_two_track(int64_t d, const float *gw, const float *gv, float lr, float b1,
+                               float b2, float c1, float c2, float eps, float ibc1, float ibc2,
+                               float *beta, float *m, float *u)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        float t1 = b1 * m[i];
+        float mi = fmaf(c1, gw[i], t1);
+        float g2 = gv[i] * gv[i];
+        float t2 = b2 * u[i];
+        float ui = fmaf(c2, g2, t2);
+        float mhat = mi * ibc1;
+        float uhat = ui * ibc2;
+        float den = sqrtf(uhat) + eps;
+        float step = mhat / den;
+        beta[i] = fmaf(-lr, step, beta[i]);
+        m[i] = mi;
+        u[i] = ui;
+    }
+}

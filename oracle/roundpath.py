@@ -49,6 +49,9 @@ def lib():
         L.agc_oracle_decode.restype = None
         L.agc_oracle_dequantize_worker.argtypes = [C.c_int64, C.c_int, C.c_int, u32p, f32p, f32p]
         L.agc_oracle_dequantize_worker.restype = None
+        L.agc_oracle_adam_two_track.argtypes = [C.c_int64, f32p, f32p, C.c_float, C.c_float, C.c_float, C.c_float,
+                                                C.c_float, C.c_float, C.c_float, C.c_float, f32p, f32p, f32p]
+        L.agc_oracle_adam_two_track.restype = None
         _lib = L
     return _lib
 
@@ -189,3 +192,23 @@ def dequantize_worker(d, b, B, codes_i, scales_i):
     lib().agc_oracle_dequantize_worker(d, b, B, _p(codes_i, C.c_uint32), _p(scales_i, C.c_float),
                                        _p(out, C.c_float))
     return out
+
+
+def adam_constants(b1, b2, step):
+    """(1-b1, 1-b2, 1/(1-b1^t), 1/(1-b2^t)) formed in double precision from the fp32 values
+    of b1, b2 and rounded to fp32 (t = step >= 1)."""
+    b1, b2 = float(np.float32(b1)), float(np.float32(b2))
+    return (np.float32(1.0 - b1), np.float32(1.0 - b2), np.float32(1.0 / (1.0 - b1 ** step)),
+            np.float32(1.0 / (1.0 - b2 ** step)))
+
+
+def adam_two_track(gw, gv, lr, b1, b2, eps, step, beta, m, u):
+    """One Adam step with first moment from gw and second moment from gv (Sec. V-E).
+    Returns updated copies (beta, m, u)."""
+    gw, gv = _c(gw, np.float32), _c(gv, np.float32)
+    beta, m, u = (np.array(x, dtype=np.float32, copy=True) for x in (beta, m, u))
+    c1, c2, ibc1, ibc2 = adam_constants(b1, b2, step)
+    lib().agc_oracle_adam_two_track(len(gw), _p(gw, C.c_float), _p(gv, C.c_float), np.float32(lr), np.float32(b1),
+                                    np.float32(b2), c1, c2, np.float32(eps), ibc1, ibc2, _p(beta, C.c_float),
+                                    _p(m, C.c_float), _p(u, C.c_float))
+    return beta, m, u

@@ -414,3 +414,35 @@ def test_block_entry_points_agree_with_whole_vector_drivers():
             wb += nw
         gb = orp.decode_block(bits, B, w, mask, cb, sb)
         assert (gb[:hi - q * 512] == gh[0, q * 512:hi]).all()
+
+
+def test_adam_two_track_against_torch_adam_and_float64():
+    """The Adam step of the two-track variant (Sec. V-E). With g_v = g_w it is plain Adam:
+    compare several steps with torch.optim.Adam (an independent library routine) and with
+    the published recursion in float64; with g_v != g_w only the second moment changes."""
+    import torch
+    rng = np.random.default_rng(4)
+    d = 1000
+    lr, b1, b2, eps = 1e-2, 0.9, 0.999, 1e-8
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    grads = [rng.standard_normal(d).astype(np.float32) * 10.0 ** rng.uniform(-3, 1) for _ in range(6)]
+    beta, m, u = beta0.copy(), np.zeros(d, np.float32), np.zeros(d, np.float32)
+    tp = torch.nn.Parameter(torch.from_numpy(beta0.copy()))
+    opt = torch.optim.Adam([tp], lr=lr, betas=(b1, b2), eps=eps)
+    b64, m64, u64 = beta0.astype(np.float64), np.zeros(d), np.zeros(d)
+    for t, g in enumerate(grads, start=1):
+        beta, m, u = orp.adam_two_track(g, g, lr, b1, b2, eps, t, beta, m, u)
+        tp.grad = torch.from_numpy(g.copy())
+        opt.step()
+        m64 = b1 * m64 + (1 - b1) * g
+        u64 = b2 * u64 + (1 - b2) * g.astype(np.float64) ** 2
+        b64 = b64 - lr * (m64 / (1 - b1 ** t)) / (np.sqrt(u64 / (1 - b2 ** t)) + eps)
+        assert np.abs(beta - tp.detach().numpy()).max() <= 2e-6 * max(1.0, np.abs(beta).max())
+        assert np.abs(beta - b64).max() <= 2e-6 * max(1.0, np.abs(b64).max())
+    # second track: only u (and through it the step) sees g_v
+    gw, gv = grads[0], grads[1]
+    z = np.zeros(d, np.float32)
+    _, m1, u1 = orp.adam_two_track(gw, gv, lr, b1, b2, eps, 1, beta0, z, z)
+    b1f, b2f = float(np.float32(b1)), float(np.float32(b2))   # the decay rates as fp32 holds them
+    assert np.allclose(m1, (1 - b1f) * gw, rtol=1e-6, atol=0)
+    assert np.allclose(u1, (1 - b2f) * gv.astype(np.float64) ** 2, rtol=1e-6, atol=0)
