@@ -163,6 +163,53 @@ int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
                const uint8_t *masks_dev, int R, const float *lr_host, float *ghat_dev,
                float *beta_dev, uint32_t *status_dev, void *cuda_stream);
 
+/* Constants of one Adam step (Kingma & Ba, 2015): step >= 1 is the iteration count t of the
+ * bias corrections 1 - beta1^t, 1 - beta2^t. */
+typedef struct agc_adam {
+    float lr, beta1, beta2, eps;
+    int64_t step;
+} agc_adam_t;
+
+/*
+ * agc_decode_two_track - two decodings of the same received messages, for adaptive
+ * optimisers (Sec. V-E): g_w = sum_i I_i w_i q_i with the plan's unbiased coefficients w
+ * feeds the first moment, g_v = sum_i I_i v_i q_i with a second coefficient vector v (the
+ * variance-reduced v* of Eq. twodec, see agc_two_track_vector) feeds the second moment; one
+ * pass over the messages, no extra communication. Optionally fused with the Adam step
+ *   m <- (1-beta1) g_w + beta1 m;   u <- (1-beta2) g_v^2 + beta2 u;
+ *   beta <- beta - lr * (m / (1-beta1^t)) / (sqrt(u / (1-beta2^t)) + eps).
+ *
+ *   codes_dev, scales_dev  device, as written by agc_encode_quantize
+ *   mask_dev   device, n bytes, 1 = arrived (one realisation)
+ *   v_host     host, n floats: the second decoding coefficients
+ *   ghat_w_dev, ghat_v_dev  device out or NULL: d fp32 each
+ *   beta_dev, m_dev, u_dev  device in/out, d fp32 each, 16-byte aligned; all three or none
+ *   adam       host; required iff beta_dev is given
+ *   status_dev as in agc_decode
+ * At least one output must be requested. Sums run over the workers in ascending order with
+ * fused multiply-adds; every step of the update is a single fp32 operation in the order
+ * written above (1-beta, 1/(1-beta^t) are formed in double precision and rounded once).
+ * Returns AGC_ERR_STATE for plans that cannot use the staged decoder (more than 2048
+ * workers, AGC_FLAG_FORCE_DIRECT). Asynchronous on the stream.
+ */
+int agc_decode_two_track(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+                         const uint8_t *mask_dev, const float *v_host, float *ghat_w_dev,
+                         float *ghat_v_dev, float *beta_dev, float *m_dev, float *u_dev,
+                         const agc_adam_t *adam, uint32_t *status_dev, void *cuda_stream);
+
+/*
+ * agc_two_track_vector - the second-moment decoder of Sec. V-E in closed form:
+ *   v_i = k Lambda / ((p_i + eta phi(b_i)) (sum_j a_ij) (1 + Lambda sum_m c_m^-1)),
+ * c_m = (p_m + eta phi(b_m)) / (1 - p_m), k partitions, phi as in agc_bit_allocate.
+ *   row_ptr, a   host CSR of the encoding matrix (n+1 row pointers, nnz coefficients)
+ *   lambda       weight of the squared bias against the variance (the paper uses 1)
+ *   v_out        host out, n floats. Workers with an empty row get 0.
+ * Host only, no CUDA.
+ */
+int agc_two_track_vector(int n, int k, const double *p, const uint8_t *bits, double phi_dim,
+                         double eta, double lambda, const int32_t *row_ptr, const float *a,
+                         float *v_out);
+
 /*
  * agc_decode_update_static - the multi-realisation fused update without any allocation.
  * (The paper has no counterpart: this entry point exists for deployment reasons only.)

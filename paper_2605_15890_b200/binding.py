@@ -22,6 +22,11 @@ AGC_CODE_SUPPORT = 1
 AGC_ERR_LIMIT = -10
 
 
+class AgcAdam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("step", C.c_int64)]
+
+
 class AgcError(RuntimeError):
     def __init__(self, code, text):
         super().__init__(f"agc error {code}: {text}")
@@ -62,6 +67,11 @@ def _load():
     L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
                                            vp, vp]
     L.agc_decode_update_static.restype = C.c_int
+    L.agc_decode_two_track.argtypes = [vp, vp, vp, vp, f32p, vp, vp, vp, vp, vp, C.POINTER(AgcAdam), vp, vp]
+    L.agc_decode_two_track.restype = C.c_int
+    L.agc_two_track_vector.argtypes = [C.c_int, C.c_int, f64p, u8p, C.c_double, C.c_double, C.c_double, i32p, f32p,
+                                       f32p]
+    L.agc_two_track_vector.restype = C.c_int
     L.agc_round_host.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, u32p, vp]
     L.agc_round_host.restype = C.c_int
     for name in ("agc_bit_allocate", "agc_bit_allocate_dp"):
@@ -185,6 +195,26 @@ def agc_decode_update_static(n_workers, d, bucket, bits, w, codes_dev, scales_de
     _check(_lib.agc_decode_update_static(n_workers, d, bucket, _hp(bits, C.c_uint8), _hp(w, C.c_float),
                                          _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
                                          _hp(lr, C.c_float), _dev(beta_dev), _stream(stream)))
+
+
+def agc_decode_two_track(plan, codes_dev, scales_dev, mask_dev, v_host, ghat_w_dev=None, ghat_v_dev=None,
+                         beta_dev=None, m_dev=None, u_dev=None, adam=None, status_dev=None, stream=None):
+    """adam: (lr, beta1, beta2, eps, step) or None."""
+    v = _np(v_host, np.float32)
+    ad = None if adam is None else AgcAdam(float(adam[0]), float(adam[1]), float(adam[2]), float(adam[3]), int(adam[4]))
+    _check(_lib.agc_decode_two_track(plan, _dev(codes_dev), _dev(scales_dev), _dev(mask_dev), _hp(v, C.c_float),
+                                     _dev(ghat_w_dev), _dev(ghat_v_dev), _dev(beta_dev), _dev(m_dev), _dev(u_dev),
+                                     None if ad is None else C.byref(ad), _dev(status_dev), _stream(stream)))
+
+
+def agc_two_track_vector(n, k, p, bits, phi_dim, row_ptr, a, eta=1.0, lam=1.0):
+    """Returns v* float32 [n] (Sec. V-E)."""
+    p, bits = _np(p, np.float64), _np(bits, np.uint8)
+    row_ptr, a = _np(row_ptr, np.int32), _np(a, np.float32)
+    v = np.zeros(n, np.float32)
+    _check(_lib.agc_two_track_vector(n, k, _hp(p, C.c_double), _hp(bits, C.c_uint8), phi_dim, eta, lam,
+                                     _hp(row_ptr, C.c_int32), _hp(a, C.c_float), _hp(v, C.c_float)))
+    return v
 
 
 def agc_round_host(plan, G_host, ld_host, rnd, mask_host, ghat_host, stream=None):

@@ -5,6 +5,7 @@
 // One warp owns one 512-coordinate pack block. Lane l holds the 16 coordinates
 // {128c + 4l + e}, i.e. stream positions 16l..16l+15 of every worker's message, so it
 // reads 16*b_i contiguous bits per worker and never needs another lane's data.
+#include <cmath>
 #include <mutex>
 
 #include "agc_internal.h"
@@ -238,17 +239,21 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 //   to   warp * 64 + (lane / 2) * 4 (odd widths: a pair of lanes shares BITS words)
 // The integer code c becomes the float 2^23 + c by OR-ing it into the mantissa of 2^23
 // (one byte permute for 8-bit codes); level = that - (2^23 + L) is exact.
-template <int BITS>
+template <int BITS, bool TWO = false>
 __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uint32_t to, int lane,
-                                                const float (&ws_row)[4], float (&acc)[16])
+                                                const float (&ws_row)[4], float (&acc)[16],
+                                                const float (&ws2_row)[4], float (&acc2)[16])
 {
     constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
     constexpr uint32_t MASK = (1u << BITS) - 1u;
     constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)(BITS >= 2 ? L : 1u)) : 2.0f;
     constexpr int NACC = (16 * BITS + 31) / 32;
-    float cstep_row[4];
+    float cstep_row[4], cstep2_row[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
+    for (int c = 0; c < 4; ++c) {
+        cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
+        cstep2_row[c] = TWO ? __fmul_rn(ws2_row[c], DSTEP) : 0.0f;
+    }
     uint32_t A[NACC + 1];
     A[NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
@@ -294,15 +299,72 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
             level = __fsub_rn(__uint_as_float(x), 8388608.0f + (float)L);                   // code - L, exact
         }
         acc[t] = __fmaf_rn(cstep_row[t >> 2], level, acc[t]);
+        if constexpr (TWO) acc2[t] = __fmaf_rn(cstep2_row[t >> 2], level, acc2[t]);
     }
 }
 
-template <int RB, bool COLLAPSED>
-__global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kernel(const AgcDecParams P)
+// Adam step on the lane's 16 coordinates of block q (Kingma & Ba, Algorithm 1) with the
+// first moment fed by gw and the second by gv (the two-track decoding of Sec. V-E); one
+// IEEE fp32 operation per step, in this order:
+//   m <- c1 * gw + b1 * m;  u <- c2 * gv^2 + b2 * u;
+//   beta <- beta - lr * (m * ibc1) / (sqrt(u * ibc2) + eps)
+__device__ __forceinline__ void adam_update16(const AgcDecParams &P, long long q, int lane, bool vec,
+                                              const float (&gw)[16], const float (&gv)[16])
 {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const long long m0 = q * AGC_BLOCK + c * 128 + 4 * lane;
+        float bt[4], mm[4], uu[4];
+        const bool full = vec && m0 + 3 < P.d;
+        if (full) {
+            const float4 x = *reinterpret_cast<const float4 *>(P.beta + m0);
+            const float4 y = *reinterpret_cast<const float4 *>(P.adam_m + m0);
+            const float4 z = *reinterpret_cast<const float4 *>(P.adam_u + m0);
+            bt[0] = x.x; bt[1] = x.y; bt[2] = x.z; bt[3] = x.w;
+            mm[0] = y.x; mm[1] = y.y; mm[2] = y.z; mm[3] = y.w;
+            uu[0] = z.x; uu[1] = z.y; uu[2] = z.z; uu[3] = z.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool in = m0 + e < P.d;
+                bt[e] = in ? P.beta[m0 + e] : 0.0f;
+                mm[e] = in ? P.adam_m[m0 + e] : 0.0f;
+                uu[e] = in ? P.adam_u[m0 + e] : 0.0f;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float mi = __fmaf_rn(P.adam_c1, gw[4 * c + e], __fmul_rn(P.adam_b1, mm[e]));
+            const float g2 = __fmul_rn(gv[4 * c + e], gv[4 * c + e]);
+            const float ui = __fmaf_rn(P.adam_c2, g2, __fmul_rn(P.adam_b2, uu[e]));
+            const float den = __fadd_rn(__fsqrt_rn(__fmul_rn(ui, P.adam_ibc2)), P.adam_eps);
+            const float step = __fdiv_rn(__fmul_rn(mi, P.adam_ibc1), den);
+            bt[e] = __fmaf_rn(-P.lr0, step, bt[e]);
+            mm[e] = mi;
+            uu[e] = ui;
+        }
+        if (full) {
+            *reinterpret_cast<float4 *>(P.beta + m0) = make_float4(bt[0], bt[1], bt[2], bt[3]);
+            *reinterpret_cast<float4 *>(P.adam_m + m0) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+            *reinterpret_cast<float4 *>(P.adam_u + m0) = make_float4(uu[0], uu[1], uu[2], uu[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (m0 + e < P.d) { P.beta[m0 + e] = bt[e]; P.adam_m[m0 + e] = mm[e]; P.adam_u[m0 + e] = uu[e]; }
+        }
+    }
+}
+
+// MODE 0: one realisation (g_hat and / or the fused update); 1: collapsed multi-realisation
+// update; 2: two-track decode (weights w and v over the same messages) with the Adam step.
+template <int RB, int MODE, int QT>
+__global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const AgcDecParams P)
+{
+    constexpr bool COLLAPSED = MODE == 1;
+    constexpr bool TWO = MODE == 2;
     extern __shared__ __align__(1024) unsigned char smem[];
     const int stages = P.stages;
-    const uint32_t stage_bytes = AGC_DEC_QT * 64u * AGC_DEC_GROUP_BITS;
+    const uint32_t stage_bytes = QT * 64u * AGC_DEC_GROUP_BITS;
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)stages * stage_bytes);
     uint64_t *empty = full + AGC_DEC_MAX_STAGES;
     volatile int *flags = reinterpret_cast<volatile int *>(empty + AGC_DEC_MAX_STAGES);  // abort x2, n_groups
@@ -311,13 +373,14 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     float *s_raw_w = reinterpret_cast<float *>(s_grp_ptr + P.n + 1);
     uint8_t *s_raw_b = reinterpret_cast<uint8_t *>(s_raw_w + P.n);
     uint8_t *s_raw_allb = s_raw_b + P.n;
+    float *s_w2 = reinterpret_cast<float *>(smem + P.w2_offset);   // second decoder of the received workers
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], AGC_DEC_QT);
+            mbar_init(&empty[s], QT);
         }
         flags[0] = 0;
         flags[1] = 0;
@@ -370,8 +433,9 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
             wk.soff = soff;
             wk.bits = b;
             wk.run = 1;
+            if (TWO) s_w2[nrecv] = P.v[i];
             s_wk[nrecv++] = wk;
-            soff += AGC_DEC_QT * 64u * b;
+            soff += QT * 64u * b;
             grp_bits += b;
             ++in_grp;
         }
@@ -380,17 +444,17 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     }
     __syncthreads();
     const int n_groups = flags[2];
-    const long long ntile = (P.nblk + AGC_DEC_QT - 1) / AGC_DEC_QT;
+    const long long ntile = (P.nblk + QT - 1) / QT;
 
-    if (warp == AGC_DEC_QT) {
+    if (warp == QT) {
         // ---------------- producer
         long long issued = 0;
         int s = 0;
         uint32_t parity = 1;
         bool ok = true;
         for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q0 = T * AGC_DEC_QT;
-            const uint32_t nq = (uint32_t)(P.nblk - q0 < AGC_DEC_QT ? P.nblk - q0 : AGC_DEC_QT);
+            const long long q0 = T * QT;
+            const uint32_t nq = (uint32_t)(P.nblk - q0 < QT ? P.nblk - q0 : QT);
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 uint32_t bytes = 0, soff = 0, wbits = 0;
@@ -414,10 +478,10 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
 #if AGC_DEC_PREFETCH
                     // the same workers' chunks of this CTA's next tile row: on their way to L2 a
                     // whole tile row ahead, so that the ring refills at L2 latency, not HBM latency
-                    const long long qn = q0 + (long long)gridDim.x * AGC_DEC_QT;
+                    const long long qn = q0 + (long long)gridDim.x * QT;
                     if (qn < P.nblk) {
-                        const uint32_t nqn = (uint32_t)(P.nblk - qn < AGC_DEC_QT ? P.nblk - qn : AGC_DEC_QT);
-                        bulk_prefetch_l2(src + (size_t)gridDim.x * AGC_DEC_QT * 64u * wbits, nqn * 64u * wbits);
+                        const uint32_t nqn = (uint32_t)(P.nblk - qn < QT ? P.nblk - qn : QT);
+                        bulk_prefetch_l2(src + (size_t)gridDim.x * QT * 64u * wbits, nqn * 64u * wbits);
                     }
 #endif
                 }
@@ -442,7 +506,7 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
         auto fetch_scales = [&](long long T, int g, float (&sc)[4 / RB]) {
 #pragma unroll
             for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
-            const long long q = T * AGC_DEC_QT + warp;
+            const long long q = T * QT + warp;
             if (T < ntile && g < n_groups && q < P.nblk) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 if (lane < nr) {
@@ -458,11 +522,13 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
         float sc_next[4 / RB];
         fetch_scales(blockIdx.x, 0, sc_next);
         for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q = T * AGC_DEC_QT + warp;
+            const long long q = T * QT + warp;
             const bool active = q < P.nblk;
-            float acc[16], b[16];
+            float acc[16], acc2[16], b[16];   // acc2: second track, unused and dropped in the other modes
 #pragma unroll
             for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) acc2[t] = 0.0f;
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 float sc[4 / RB];
@@ -471,7 +537,7 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 if (g + 1 < n_groups) fetch_scales(T, g + 1, sc_next);
                 else fetch_scales(T + gridDim.x, 0, sc_next);
                 // parameters of the block: read early, used after the last group
-                if (g == n_groups - 1 && P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
+                if (!TWO && g == n_groups - 1 && P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
                 ok = mbar_wait(&full[s], parity, flags);
                 if (!ok) break;
                 if (active) {
@@ -484,12 +550,18 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     for (int j = 0; j < run; ++j) {                                                             \
         const float weight = s_wk[r0 + r + j].weight;                                           \
         const uint32_t chunk = stage + s_wk[r0 + r + j].soff;                                   \
-        float ws_row[4];                                                                        \
+        const float weight2 = TWO ? s_w2[r0 + r + j] : 0.0f;                                    \
+        float ws_row[4], ws2_row[4];                                                            \
         _Pragma("unroll") for (int bk = 0; bk < 4 / RB; ++bk) {                                 \
-            const float ws = __fmul_rn(weight, __shfl_sync(0xffffffffu, sc[bk], r + j));        \
-            _Pragma("unroll") for (int cc = 0; cc < RB; ++cc) ws_row[bk * RB + cc] = ws;        \
+            const float S = __shfl_sync(0xffffffffu, sc[bk], r + j);                            \
+            const float ws = __fmul_rn(weight, S);                                              \
+            const float ws2 = TWO ? __fmul_rn(weight2, S) : 0.0f;                               \
+            _Pragma("unroll") for (int cc = 0; cc < RB; ++cc) {                                 \
+                ws_row[bk * RB + cc] = ws;                                                      \
+                ws2_row[bk * RB + cc] = ws2;                                                    \
+            }                                                                                   \
         }                                                                                       \
-        ring_add_worker<B>(chunk, tl, to, lane, ws_row, acc);                                   \
+        ring_add_worker<B, TWO>(chunk, tl, to, lane, ws_row, acc, ws2_row, acc2);               \
     }
                         switch (bits) {
                             case 1: AGC_DEC_RUN(1) break;
@@ -509,7 +581,11 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
                 if (lane == 0) mbar_arrive(&empty[s]);
                 if (++s == stages) { s = 0; parity ^= 1u; }
             }
-            if (ok && active) {
+            if (ok && active && TWO) {
+                if (P.ghat) store16(P.ghat, q, lane, P.d, vec, acc);
+                if (P.ghat_v) store16(P.ghat_v, q, lane, P.d, vec, acc2);
+                if (P.beta) adam_update16(P, q, lane, vec, acc, acc2);
+            } else if (ok && active) {
                 if (n_groups == 0 && P.beta) load16(P.beta, q, lane, P.d, vec, b);
                 if (COLLAPSED) {
 #pragma unroll
@@ -530,14 +606,41 @@ __global__ void __launch_bounds__((AGC_DEC_QT + 1) * 32, 1) agc_decode_ring_kern
     if (threadIdx.x == 0 && (flags[0] || flags[1]) && P.status) atomicOr(P.status, AGC_STATUS_TIMEOUT);
 }
 
-template <bool COLLAPSED>
+template <int MODE, int QT>
 cudaError_t launch_ring(const AgcDecParams &P, int grid, size_t smem, cudaStream_t stream)
 {
-    const int threads = (AGC_DEC_QT + 1) * 32;
-    if (P.rows_per_bucket == 4) agc_decode_ring_kernel<4, COLLAPSED><<<grid, threads, smem, stream>>>(P);
-    else if (P.rows_per_bucket == 2) agc_decode_ring_kernel<2, COLLAPSED><<<grid, threads, smem, stream>>>(P);
-    else agc_decode_ring_kernel<1, COLLAPSED><<<grid, threads, smem, stream>>>(P);
+    const int threads = (QT + 1) * 32;
+    if (P.rows_per_bucket == 4) agc_decode_ring_kernel<4, MODE, QT><<<grid, threads, smem, stream>>>(P);
+    else if (P.rows_per_bucket == 2) agc_decode_ring_kernel<2, MODE, QT><<<grid, threads, smem, stream>>>(P);
+    else agc_decode_ring_kernel<1, MODE, QT><<<grid, threads, smem, stream>>>(P);
     return cudaGetLastError();
+}
+
+// Shared-memory layout of the ring decoder for a tile of QT blocks: stages, then the tables.
+// Returns the ring depth (0: does not fit) and the total size / offset of the second weights.
+template <int QT>
+int ring_layout(int n, int smem_optin, size_t *smem_out, uint32_t *w2_offset)
+{
+    const size_t stage_bytes = size_t(QT) * 64 * AGC_DEC_GROUP_BITS;
+    size_t tail = (2 * AGC_DEC_MAX_STAGES + 2) * sizeof(uint64_t) + sizeof(AgcDecWorker) * size_t(n) +
+                  sizeof(int32_t) * (size_t(n) + 1) + 6 * size_t(n);
+    tail = (tail + 15) & ~size_t(15);
+    const size_t w2_rel = tail;
+    tail += sizeof(float) * size_t(n) + 16;
+    if (size_t(smem_optin) < tail + 2 * stage_bytes) return 0;
+    long long stages = (long long)((size_t(smem_optin) - tail) / stage_bytes);
+    if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
+    *smem_out = size_t(stages) * stage_bytes + tail;
+    *w2_offset = uint32_t(size_t(stages) * stage_bytes + w2_rel);
+    return int(stages);
+}
+
+template <int MODE, int QT>
+bool ring_set_smem(int smem)
+{
+    return cudaFuncSetAttribute(agc_decode_ring_kernel<4, MODE, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) == cudaSuccess &&
+           cudaFuncSetAttribute(agc_decode_ring_kernel<2, MODE, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) == cudaSuccess &&
+           cudaFuncSetAttribute(agc_decode_ring_kernel<1, MODE, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) == cudaSuccess;
 }
 
 template <bool COLLAPSED>
@@ -574,6 +677,7 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     P.lr = plan->d_lr;
     P.status = status;
     P.stages = plan->dec_stages;
+    P.w2_offset = plan->dec_w2_offset;
     const bool collapsed = R > 1 && beta && !ghat;
     if (beta && R > 1) {
         if (cudaMemcpyAsync(plan->d_lr, lr_host, sizeof(float) * R, cudaMemcpyHostToDevice, stream) != cudaSuccess)
@@ -588,14 +692,14 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
         const long long ntile = (plan->nblk + AGC_DEC_QT - 1) / AGC_DEC_QT;
         const int grid = (int)(ntile < plan->sm_count ? ntile : plan->sm_count);
         if (collapsed) {
-            if (launch_ring<true>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
+            if (launch_ring<1, AGC_DEC_QT>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
         } else {
             // one launch per realisation, in order: realisation r sees beta after r - 1
             for (int r = 0; r < R; ++r) {
                 P.masks = masks + (size_t)r * plan->n;
                 P.ghat = ghat ? ghat + (size_t)r * plan->d : nullptr;
                 P.lr0 = (beta && lr_host) ? lr_host[r] : 0.0f;
-                if (launch_ring<false>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
+                if (launch_ring<0, AGC_DEC_QT>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
             }
         }
         return AGC_OK;
@@ -606,29 +710,68 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
 }
 
-// Decide whether the plan decodes with the ring kernel and size its shared memory.
+// Decide whether the plan decodes with the ring kernels and size their shared memory.
 int agc_decode_prepare(agc_plan *plan, int smem_optin)
 {
     plan->dec_ring = false;
     if ((plan->flags & AGC_FLAG_FORCE_DIRECT) || plan->n > AGC_DEC_RING_MAX_WORKERS) return AGC_OK;
-    const size_t stage_bytes = size_t(AGC_DEC_QT) * 64 * AGC_DEC_GROUP_BITS;
-    const size_t tail = (2 * AGC_DEC_MAX_STAGES + 2) * sizeof(uint64_t) + sizeof(AgcDecWorker) * size_t(plan->n) +
-                        sizeof(int32_t) * (size_t(plan->n) + 1) + 6 * size_t(plan->n) + 16;
-    if (size_t(smem_optin) < tail + 2 * stage_bytes) return AGC_OK;
-    long long stages = (long long)((size_t(smem_optin) - tail) / stage_bytes);
-    if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
-    plan->dec_stages = int(stages);
-    plan->dec_smem = size_t(stages) * stage_bytes + tail;
-    const int smem = int(plan->dec_smem);
-    if (cudaFuncSetAttribute(agc_decode_ring_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_ring_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_ring_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_ring_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_ring_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_ring_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    plan->dec_stages = ring_layout<AGC_DEC_QT>(plan->n, smem_optin, &plan->dec_smem, &plan->dec_w2_offset);
+    plan->dec2_stages = ring_layout<AGC_DEC_QT2>(plan->n, smem_optin, &plan->dec2_smem, &plan->dec2_w2_offset);
+    if (plan->dec_stages < 2 || plan->dec2_stages < 2) return AGC_OK;
+    if (!ring_set_smem<0, AGC_DEC_QT>(int(plan->dec_smem)) || !ring_set_smem<1, AGC_DEC_QT>(int(plan->dec_smem)) ||
+        !ring_set_smem<2, AGC_DEC_QT2>(int(plan->dec2_smem)))
         return AGC_ERR_CUDA;
     plan->dec_ring = true;
     return AGC_OK;
+}
+
+int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *scales, const uint8_t *mask,
+                                const float *v_host, float *ghat_w, float *ghat_v, float *beta, float *m,
+                                float *u, const agc_adam_t *adam, uint32_t *status, cudaStream_t stream)
+{
+    if (!plan->dec_ring) return AGC_ERR_STATE;
+    if (cudaMemcpyAsync(plan->d_v, v_host, sizeof(float) * plan->n, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    AgcDecParams P;
+    P.bits = plan->d_bits;
+    P.w = plan->d_w;
+    P.word_off = plan->d_word_off;
+    P.codes = static_cast<const uint32_t *>(codes);
+    P.scales = scales;
+    P.masks = mask;
+    P.weff = nullptr;
+    P.ghat = ghat_w;
+    P.beta = beta;
+    P.d = plan->d;
+    P.nblk = plan->nblk;
+    P.nb = plan->nb;
+    P.n = plan->n;
+    P.R = 1;
+    P.rows_per_bucket = plan->bucket / 128;
+    P.lr0 = 0.0f;
+    P.lr = nullptr;
+    P.status = status;
+    P.stages = plan->dec2_stages;
+    P.w2_offset = plan->dec2_w2_offset;
+    P.v = plan->d_v;
+    P.ghat_v = ghat_v;
+    P.adam_m = m;
+    P.adam_u = u;
+    if (beta) {
+        // constants of the step, formed in double precision and rounded once
+        const double b1 = double(adam->beta1), b2 = double(adam->beta2);
+        P.lr0 = adam->lr;
+        P.adam_b1 = adam->beta1;
+        P.adam_b2 = adam->beta2;
+        P.adam_c1 = float(1.0 - b1);
+        P.adam_c2 = float(1.0 - b2);
+        P.adam_eps = adam->eps;
+        P.adam_ibc1 = float(1.0 / (1.0 - std::pow(b1, double(adam->step))));
+        P.adam_ibc2 = float(1.0 / (1.0 - std::pow(b2, double(adam->step))));
+    }
+    const long long ntile = (plan->nblk + AGC_DEC_QT2 - 1) / AGC_DEC_QT2;
+    const int grid = (int)(ntile < plan->sm_count ? ntile : plan->sm_count);
+    return launch_ring<2, AGC_DEC_QT2>(P, grid, plan->dec2_smem, stream) == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------ allocation-free update

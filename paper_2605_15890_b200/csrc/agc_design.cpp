@@ -342,3 +342,25 @@ extern "C" int agc_code_build(int n, int k, const double *p, const uint8_t *bits
     }
     return AGC_OK;
 }
+
+extern "C" int agc_two_track_vector(int n, int k, const double *p, const uint8_t *bits, double phi_dim,
+                                    double eta, double lambda, const int32_t *row_ptr, const float *a,
+                                    float *v_out)
+{
+    if (n < 1 || k < 1 || !p || !bits || !row_ptr || !a || !v_out || !(phi_dim > 0.0) || !(eta > 0.0) ||
+        !(lambda > 0.0))
+        return AGC_ERR_ARG;
+    double sum_cinv = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (!(p[i] >= 0.0 && p[i] < 1.0)) return AGC_ERR_PROB;
+        if (bits[i] < 1 || bits[i] > 8) return AGC_ERR_BITS;
+        sum_cinv += (1.0 - p[i]) / (p[i] + phi_of(bits[i], phi_dim, eta));
+    }
+    for (int i = 0; i < n; ++i) {
+        double row = 0.0;
+        for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e) row += double(a[e]);
+        const double den = (p[i] + phi_of(bits[i], phi_dim, eta)) * row * (1.0 + lambda * sum_cinv);
+        v_out[i] = row > 0.0 ? float(double(k) * lambda / den) : 0.0f;
+    }
+    return AGC_OK;
+}

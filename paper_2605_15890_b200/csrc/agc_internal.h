@@ -26,6 +26,7 @@
 #define AGC_DEC_GROUP_BITS 32  // cap on sum of b_i over a worker group: stage = QT * 64 * this bytes
 #endif
 #define AGC_DEC_MAX_STAGES 8
+#define AGC_DEC_QT2 23         // consumer warps of the two-track decoder (two accumulator sets: 80 registers)
 #define AGC_DEC_RING_MAX_WORKERS 2048  // above this the per-worker tables no longer fit shared memory
 #define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
 #define AGC_STATIC_MAX_R 4096
@@ -98,6 +99,12 @@ struct AgcDecParams {
     const float *lr;        // device, R learning rates (per-realisation mode with beta)
     uint32_t *status = nullptr;  // AGC_STATUS_* bits are OR-ed into it (ring kernel), may be NULL
     int stages = 0;              // ring depth of the ring kernel
+    uint32_t w2_offset = 0;      // byte offset of the second-decoder array in shared memory
+    // two-track decode
+    const float *v = nullptr;    // n second decoding coefficients
+    float *ghat_v = nullptr;     // d or NULL
+    float *adam_m = nullptr, *adam_u = nullptr;
+    float adam_b1 = 0.f, adam_b2 = 0.f, adam_c1 = 0.f, adam_c2 = 0.f, adam_eps = 0.f, adam_ibc1 = 0.f, adam_ibc2 = 0.f;
 };
 
 struct agc_plan {
@@ -120,6 +127,10 @@ struct agc_plan {
     bool dec_ring = false;
     int dec_stages = 0;
     size_t dec_smem = 0;
+    int dec2_stages = 0;
+    size_t dec2_smem = 0;
+    uint32_t dec_w2_offset = 0, dec2_w2_offset = 0;
+    float *d_v = nullptr;
     // device tables
     int32_t *d_row_ptr = nullptr, *d_col_idx = nullptr;
     float *d_a = nullptr, *d_w = nullptr;
@@ -144,3 +155,6 @@ int agc_launch_encode(agc_plan *plan, const float *G, long long ld, uint64_t rou
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
                       int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
                       cudaStream_t stream);
+int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *scales, const uint8_t *mask,
+                                const float *v_host, float *ghat_w, float *ghat_v, float *beta, float *m,
+                                float *u, const agc_adam_t *adam, uint32_t *status, cudaStream_t stream);

@@ -89,7 +89,7 @@ void free_device(agc_plan *p)
     cudaFree(p->d_row_ptr); cudaFree(p->d_col_idx); cudaFree(p->d_a); cudaFree(p->d_w);
     cudaFree(p->d_bits); cudaFree(p->d_wdesc); cudaFree(p->d_edesc); cudaFree(p->d_word_off);
     cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_op_ptr); cudaFree(p->d_ops); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
-    cudaFree(p->d_weff); cudaFree(p->d_lr);
+    cudaFree(p->d_weff); cudaFree(p->d_lr); cudaFree(p->d_v);
     cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
     cudaFree(p->h_mask); cudaFree(p->h_status);
 }
@@ -214,6 +214,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc) rc = upload(&pl->d_grp_wk_ptr, grp_wk_ptr);
     if (!rc) rc = upload(&pl->d_grp_workers, grp_workers);
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
+    if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_v), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_lr), sizeof(float) * AGC_MAX_R) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc) rc = agc_encode_prepare(pl);
     if (!rc) rc = agc_decode_prepare(pl, smem_optin);
@@ -272,6 +273,24 @@ extern "C" int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *
         return AGC_ERR_ALIGN;
     return agc_launch_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host, ghat_dev, beta_dev, status_dev,
                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int agc_decode_two_track(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+                                    const uint8_t *mask_dev, const float *v_host, float *ghat_w_dev,
+                                    float *ghat_v_dev, float *beta_dev, float *m_dev, float *u_dev,
+                                    const agc_adam_t *adam, uint32_t *status_dev, void *cuda_stream)
+{
+    if (!plan || !codes_dev || !scales_dev || !mask_dev || !v_host) return AGC_ERR_ARG;
+    if (!ghat_w_dev && !ghat_v_dev && !beta_dev) return AGC_ERR_ARG;
+    if ((beta_dev != nullptr) != (m_dev != nullptr) || (beta_dev != nullptr) != (u_dev != nullptr)) return AGC_ERR_ARG;
+    if (beta_dev && (!adam || adam->step < 1 || !(adam->beta1 >= 0.0f && adam->beta1 < 1.0f) ||
+                     !(adam->beta2 >= 0.0f && adam->beta2 < 1.0f)))
+        return AGC_ERR_ARG;
+    const void *ptrs[] = {codes_dev, ghat_w_dev, ghat_v_dev, beta_dev, m_dev, u_dev};
+    for (const void *ptr : ptrs)
+        if (ptr && (reinterpret_cast<uintptr_t>(ptr) & 15)) return AGC_ERR_ALIGN;
+    return agc_launch_decode_two_track(plan, codes_dev, scales_dev, mask_dev, v_host, ghat_w_dev, ghat_v_dev, beta_dev,
+                                       m_dev, u_dev, adam, status_dev, static_cast<cudaStream_t>(cuda_stream));
 }
 
 extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_host, uint64_t round,

@@ -392,3 +392,46 @@ def test_config4_least_squares_descent_in_lock_step(agc, torch):
     ses.close()
     assert losses[-1] < 0.05 * losses[0]
     assert min(losses) == min(losses[-50:]) or losses[-1] < 1.5 * min(losses)
+
+
+@pytest.mark.parametrize("B,d", [(512, 5000), (128, 70_001)])
+def test_two_track_decode_and_adam_steps(agc, torch, B, d):
+    """Sec. V-E: the same messages decoded with w (first moment) and with v* (second moment)
+    in one pass, fused with the Adam step; three rounds against the oracle, bit for bit."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(B + d)
+    n = k = 12
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B)
+    v = agc.agc_two_track_vector(n, k, p, bits, float(B), rp, a)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=5, flags=agc.AGC_FLAG_ALLOW_1BIT)
+    ld = (d + 3) // 4 * 4
+    lr, b1, b2, eps = 1e-2, 0.9, 0.999, 1e-8
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    beta = torch.from_numpy(beta0.copy()).cuda()
+    m = torch.zeros(d, dtype=torch.float32, device="cuda")
+    u = torch.zeros(d, dtype=torch.float32, device="cuda")
+    gw = torch.empty(d, dtype=torch.float32, device="cuda")
+    gv = torch.empty(d, dtype=torch.float32, device="cuda")
+    ob, om, ou = beta0.copy(), np.zeros(d, np.float32), np.zeros(d, np.float32)
+    for t in range(1, 4):
+        G_host = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 1)).astype(np.float32)
+        G = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+        G[:, :d] = torch.from_numpy(G_host)
+        mask = (rng.random(n) >= p).astype(np.uint8)
+        ses.encode(G, t)
+        agc.agc_decode_two_track(ses.plan, ses.codes, ses.scales, torch.from_numpy(mask).cuda(), v, gw, gv, beta, m, u,
+                                 adam=(lr, b1, b2, eps, t), status_dev=ses.status)
+        torch.cuda.synchronize()
+        oc, osc, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 5, t, G_host)
+        ogw, _ = orp.decode(d, bits, B, w, mask[None], oc, osc)
+        ogv, _ = orp.decode(d, bits, B, v, mask[None], oc, osc)
+        ob, om, ou = orp.adam_two_track(ogw[0], ogv[0], lr, b1, b2, eps, t, ob, om, ou)
+        assert (gw.cpu().numpy().view(np.uint32) == ogw[0].view(np.uint32)).all()
+        assert (gv.cpu().numpy().view(np.uint32) == ogv[0].view(np.uint32)).all()
+        assert (m.cpu().numpy().view(np.uint32) == om.view(np.uint32)).all()
+        assert (u.cpu().numpy().view(np.uint32) == ou.view(np.uint32)).all()
+        assert (beta.cpu().numpy().view(np.uint32) == ob.view(np.uint32)).all()
+    assert int(ses.status.item()) == 0
+    ses.close()

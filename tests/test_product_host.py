@@ -121,3 +121,21 @@ def test_plan_validation_rejects_bad_input_before_any_gpu_work():
             agc.agc_plan_create(2, 2, args["d"], args["rp"], args["ci"], args["a"], args["w"], args["p"],
                                 args["bits"], args["bucket"], 0, 0)
         assert e.value.code == code, kw
+
+
+def test_two_track_vector_against_oracle():
+    """v* of Sec. V-E from the library against the float64 oracle (itself pinned as the
+    minimiser of Eq. twodec)."""
+    rng = np.random.default_rng(12)
+    for n, k in [(4, 4), (7, 12), (16, 16)]:
+        p = rng.uniform(0.02, 0.5, n)
+        bits = rng.integers(2, 9, n).astype(np.uint8)
+        alpha = od.interval_alpha(od.optimal_row_sums(p, bits, k, 256), k)
+        rp, ci, vals = od.alpha_to_csr(alpha)
+        A = np.zeros((n, k))
+        for i in range(n):
+            A[i, ci[rp[i]:rp[i + 1]]] = vals[rp[i]:rp[i + 1]].astype(np.float32)
+        for lam in (0.5, 1.0, 4.0):
+            v = agc.agc_two_track_vector(n, k, p, bits, 256.0, rp, vals.astype(np.float32), lam=lam)
+            want = od.two_track_decoder(A, p, bits, 256, lam=lam)
+            assert np.allclose(v, want, rtol=2e-6, atol=0)
