@@ -205,6 +205,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-two-track", action="store_true")
     ap.add_argument("--d", type=int, default=0, help="override the number of coordinates (profiling on a small case)")
     args = ap.parse_args()
     wl = workload(args.workload)
@@ -288,6 +289,24 @@ def main():
     step_ms, k1_ms, k2_ms = sharding.max_over_ranks([step_ms, k1_ms, k2_ms], device=dev)
     value = world * wl.d / (step_ms * 1e-3)
 
+    # the two-track decode + Adam step (Sec. V-E) on the same messages: timed apart, not part of the step
+    tt_ms = None
+    if R == 1 and not args.no_two_track:
+        v2 = agc.agc_two_track_vector(wl.n, wl.k, wl.p, bits, float(bucket), rp, a)
+        m_t = torch.zeros(wl.d, dtype=torch.float32, device=dev)
+        u_t = torch.zeros(wl.d, dtype=torch.float32, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 30
+        for it in range(reps + 3):
+            if it == 3:
+                e0.record()
+            agc.agc_decode_two_track(ses.plan, ses.codes, ses.scales, masks_all[it % n_masks, 0], v2, None, None,
+                                     beta, m_t, u_t, adam=(1e-3, 0.9, 0.999, 1e-8, it + 1), status_dev=ses.status)
+        e1.record()
+        torch.cuda.synchronize()
+        tt_ms = sharding.max_over_ranks([e0.elapsed_time(e1) / reps], device=dev)[0]
+        del m_t, u_t
+
     # end to end through the host-buffer entry point (pinned host memory, copies timed)
     e2e = None
     if not args.no_e2e:
@@ -318,7 +337,7 @@ def main():
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": workload_config(wl, bits, bucket, l2_note),
                 "kernels": {"encode_quantize_ms": k1_ms, "decode_update_ms": k2_ms, "staged_tma": bool(ses.uses_tma),
-                            "status_bits": status,
+                            "status_bits": status, "two_track_adam_ms": tt_ms,
                             "decode_GBs": k2_algorithmic_bytes(wl, bits, bucket, masks_all, wl.p) / (k2_ms * 1e-3) / 1e9},
                 "roofline": {"bound": "hbm", "kernel": "agc_encode_staged_kernel" if ses.uses_tma else "agc_encode_direct_kernel",
                              "achieved": achieved, "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
