@@ -378,3 +378,81 @@ void agc_oracle_adam_two_track(int64_t d, const float *gw, const float *gv, floa
         u[i] = ui;
     }
 }
+
+/* ---- the paper's main formulation: ONE l2 norm per worker and round (Eq. quant_def with
+ * ||x||_2 over all d coordinates; the bucket-wise variant above is its extension). ----
+ *
+ * Summation order of the global sum of squares (the paper is silent): each pack block's
+ * 512 squares are summed as a 512-bucket (bucket_sumsq), then the per-block sums go through
+ * the pairwise tree in block order, level by level: entry t of the next level is
+ * v[2t] + v[2t+1], a last entry without partner is added to +0 (the same as a balanced tree
+ * over the sums padded with +0 to a power of two). */
+/*
+ * Encode + quantise + pack with the global norm. Same wire format as the bucketed path;
+ * scales has ONE entry per worker. A worker whose sum of squares is below the smallest
+ * normal number or not finite is sent as zero codes with scale 0.
+ */
+uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_t *row_ptr,
+                                           const int32_t *col_idx, const float *a,
+                                           const uint8_t *bits, uint64_t seed, uint64_t round,
+                                           const float *G, int64_t ld, uint32_t *codes,
+                                           float *scales, float *x_out)
+{
+    const int64_t nblk = agc_oracle_num_blocks(d);
+    uint32_t status = 0;
+    float *x = (float *)malloc((size_t)nblk * AGC_BLOCK * sizeof(float));
+    float *part = (float *)malloc((size_t)nblk * sizeof(float));
+    int64_t woff = 0;
+    (void)k;
+    for (int i = 0; i < n; ++i) {
+        const int b = bits[i];
+        /* Sec. II-A: f_i, ascending partitions, fp32 fma chain; zero beyond d */
+        for (int64_t m = 0; m < nblk * AGC_BLOCK; ++m) {
+            float acc = 0.0f;
+            if (m < d)
+                for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                    acc = fmaf(a[e], G[(int64_t)col_idx[e] * ld + m], acc);
+            x[m] = acc;
+        }
+        if (x_out) memcpy(x_out + (int64_t)i * d, x, (size_t)d * sizeof(float));
+        for (int64_t q = 0; q < nblk; ++q) part[q] = bucket_sumsq(x + q * AGC_BLOCK, AGC_BLOCK);
+        /* shrinking tree: level by level over the current length */
+        int64_t len = nblk;
+        while (len > 1) {
+            int64_t half = (len + 1) / 2;
+            for (int64_t t = 0; t < half; ++t)
+                part[t] = part[2 * t] + (2 * t + 1 < len ? part[2 * t + 1] : 0.0f);
+            len = half;
+        }
+        float sumsq = part[0];
+        int finite = (sumsq == sumsq) && (sumsq != INFINITY);
+        int flushed = !(finite && sumsq >= 1.17549435e-38f);
+        if (!finite) status |= AGC_ORACLE_STATUS_NONFINITE;
+        float S = flushed ? 0.0f : sqrtf(sumsq);
+        scales[i] = S;
+        float inv = flushed ? 0.0f : agc_oracle_inv_scale(S, b);
+        uint32_t *words = codes + woff;
+        memset(words, 0, (size_t)nblk * 16 * b * sizeof(uint32_t));
+        for (int64_t q = 0; q < nblk; ++q)
+            for (int o = 0; o < AGC_BLOCK; ++o) {
+                int pos = stream_pos_in_block(o);
+                uint32_t code;
+                if (flushed) {
+                    code = zero_code(b);
+                } else {
+                    uint32_t u = agc_oracle_uniform15(seed, round, (uint32_t)i,
+                                                      (uint64_t)q * AGC_BLOCK + (uint64_t)pos);
+                    code = agc_oracle_quantize_one(x[q * AGC_BLOCK + o], inv, b, u);
+                    if (code > 2u * zero_code(b) + (b == 1 ? 1u : 0u)) status |= AGC_ORACLE_STATUS_RANGE;
+                    code &= (1u << b) - 1u;
+                }
+                int bit = pos * b;
+                uint32_t *w = words + q * 16 * b;
+                w[bit >> 5] |= code << (bit & 31);
+                if ((bit & 31) + b > 32) w[(bit >> 5) + 1] |= code >> (32 - (bit & 31));
+            }
+        woff += nblk * 16 * b;
+    }
+    free(x); free(part);
+    return status;
+}

@@ -49,6 +49,9 @@ def lib():
         L.agc_oracle_decode.restype = None
         L.agc_oracle_dequantize_worker.argtypes = [C.c_int64, C.c_int, C.c_int, u32p, f32p, f32p]
         L.agc_oracle_dequantize_worker.restype = None
+        L.agc_oracle_encode_quantize_global.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_uint64,
+                                                        C.c_uint64, f32p, C.c_int64, u32p, f32p, f32p]
+        L.agc_oracle_encode_quantize_global.restype = C.c_uint32
         L.agc_oracle_adam_two_track.argtypes = [C.c_int64, f32p, f32p, C.c_float, C.c_float, C.c_float, C.c_float,
                                                 C.c_float, C.c_float, C.c_float, C.c_float, f32p, f32p, f32p]
         L.agc_oracle_adam_two_track.restype = None
@@ -212,3 +215,30 @@ def adam_two_track(gw, gv, lr, b1, b2, eps, step, beta, m, u):
                                     np.float32(b2), c1, c2, np.float32(eps), ibc1, ibc2, _p(beta, C.c_float),
                                     _p(m, C.c_float), _p(u, C.c_float))
     return beta, m, u
+
+
+def encode_quantize_global(row_ptr, col_idx, a, bits, seed, rnd, G, d=None, want_x=False):
+    """Encode + quantise + pack with ONE l2 norm per worker (the paper's main formulation).
+    Returns (codes uint32, scales float32 [n], status, x or None)."""
+    G = np.asarray(G)
+    assert G.dtype == np.float32 and G.ndim == 2 and G.strides[1] == 4
+    k = G.shape[0]
+    d = G.shape[1] if d is None else d
+    ld = G.strides[0] // 4
+    row_ptr, col_idx = _c(row_ptr, np.int32), _c(col_idx, np.int32)
+    a, bits = _c(a, np.float32), _c(bits, np.uint8)
+    n = len(bits)
+    off = worker_word_offsets(d, bits)
+    codes = np.zeros(int(off[-1]), np.uint32)
+    scales = np.zeros(n, np.float32)
+    x = np.zeros((n, d), np.float32) if want_x else None
+    st = lib().agc_oracle_encode_quantize_global(n, k, d, _p(row_ptr, C.c_int32), _p(col_idx, C.c_int32),
+                                                 _p(a, C.c_float), _p(bits, C.c_uint8), seed, rnd,
+                                                 _p(G, C.c_float), ld, _p(codes, C.c_uint32),
+                                                 _p(scales, C.c_float), _p(x, C.c_float))
+    return codes, scales, int(st), x
+
+
+def expand_global_scales(scales, d):
+    """The per-worker global scales as an (n, nblk) array for decode() with B = 512."""
+    return np.repeat(np.asarray(scales, np.float32)[:, None], num_blocks(d), axis=1)

@@ -446,3 +446,56 @@ def test_adam_two_track_against_torch_adam_and_float64():
     b1f, b2f = float(np.float32(b1)), float(np.float32(b2))   # the decay rates as fp32 holds them
     assert np.allclose(m1, (1 - b1f) * gw, rtol=1e-6, atol=0)
     assert np.allclose(u1, (1 - b2f) * gv.astype(np.float64) ** 2, rtol=1e-6, atol=0)
+
+
+def test_global_norm_encoder_pins():
+    """The paper's main formulation (Sec. II-B, Eq. quant_def with ||x||_2 over all d). (i) For
+    d <= 512 there is one block and one bucket: codes and scale must equal the bucket-wise
+    path with B = 512 bit for bit; (ii) the scale is the l2 norm of f_i (float64) to fp32
+    accuracy; (iii) a zero worker is sent as zero codes with scale 0; (iv) E[Q(x)] = x by
+    Monte-Carlo over rounds, error shrinking like 1/sqrt(rounds)."""
+    rng = np.random.default_rng(21)
+    n = k = 4
+    bits = np.array([2, 3, 5, 8], np.uint8)
+    rp = np.arange(n + 1, dtype=np.int32)
+    ci = np.arange(n, dtype=np.int32)
+    a = np.ones(n, np.float32)
+    # (i)
+    for d in (1, 77, 512):
+        G = rng.standard_normal((k, d)).astype(np.float32)
+        c1, s1, st1, _ = orp.encode_quantize_global(rp, ci, a, bits, 3, 5, G)
+        c2, s2, st2, _ = orp.encode_quantize(rp, ci, a, bits, 512, 3, 5, G)
+        assert st1 == 0 and st2 == 0
+        assert (c1 == c2).all() and (s1.view(np.uint32) == s2[:, 0].view(np.uint32)).all()
+    # (ii), (iii)
+    d = 512 * 37 + 123
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-3, 2, (k, 1))).astype(np.float32)
+    G[2] = 0.0
+    codes, scales, st, x = orp.encode_quantize_global(rp, ci, a, bits, 3, 5, G, want_x=True)
+    assert st == 0
+    want = np.sqrt((x.astype(np.float64) ** 2).sum(axis=1))
+    assert np.allclose(scales, want, rtol=3e-6, atol=0) and scales[2] == 0.0
+    off = orp.worker_word_offsets(d, bits)
+    q2 = orp.dequantize_worker(d, int(bits[2]), 512, codes[off[2]:off[3]], np.zeros(orp.num_blocks(d), np.float32))
+    assert (q2 == 0).all()
+    # every code inside its range: |x| <= S for each coordinate
+    for i in (0, 1, 3):
+        qi = orp.dequantize_worker(d, int(bits[i]), 512, codes[off[i]:off[i + 1]],
+                                   np.full(orp.num_blocks(d), scales[i], np.float32))
+        L = (1 << (int(bits[i]) - 1)) - 1
+        assert np.abs(qi - x[i]).max() <= scales[i] / L * 1.0001
+    # (iv)
+    d = 700
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    acc = np.zeros((n, d))
+    rounds = 2000
+    for t in range(rounds):
+        codes, scales, _, x = orp.encode_quantize_global(rp, ci, a, bits, 9, t, G, want_x=True)
+        off = orp.worker_word_offsets(d, bits)
+        for i in range(n):
+            acc[i] += orp.dequantize_worker(d, int(bits[i]), 512, codes[off[i]:off[i + 1]],
+                                            np.full(orp.num_blocks(d), scales[i], np.float32))
+    for i in range(n):
+        L = (1 << (int(bits[i]) - 1)) - 1
+        sigma = scales[i] / L / 2.0 / np.sqrt(rounds)       # per-coordinate std of the mean is at most this
+        assert np.abs(acc[i] / rounds - x[i]).max() <= 6.0 * sigma
