@@ -48,6 +48,8 @@ def measured_hbm_peak():
 def k1_algorithmic_bytes(wl, bits, bucket):
     """Partitions read once + packed codes + scales written (per launch)."""
     nblk = (wl.d + 511) // 512
+    if bucket == 0:   # global norm: the partial gradients are read twice, one scale per worker
+        return 8 * wl.k * wl.d + int(sum(4 * 16 * int(b) * nblk for b in bits)) + 4 * wl.n
     nb = (wl.d + bucket - 1) // bucket
     return 4 * wl.k * wl.d + int(sum(4 * 16 * int(b) * nblk for b in bits)) + 4 * wl.n * nb
 
@@ -57,7 +59,7 @@ def k2_algorithmic_bytes(wl, bits, bucket, masks_all, p):
     workers with a non-zero effective weight when R realisations are collapsed) read once,
     parameters read and written."""
     nblk = (wl.d + 511) // 512
-    nb = (wl.d + bucket - 1) // bucket
+    nb = (wl.d + bucket - 1) // bucket if bucket else 1
     m = masks_all.cpu().numpy().astype(bool)          # rounds x R x n
     used = m.any(axis=1)                              # rounds x n
     per_worker = np.array([64 * int(b) * nblk + 4 * nb for b in bits], np.float64)
@@ -108,6 +110,19 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def oracle_round(orp, code, bits, bucket, seed, t, G, d, mask, lr, beta):
+    """One round of the oracle: encode + quantise + pack, then decode + update (returns beta)."""
+    rp, ci, a, w = code
+    if bucket:
+        c, s, _, _ = orp.encode_quantize(rp, ci, a, bits, bucket, seed, t, G, d=d)
+        B = bucket
+    else:
+        c, s0, _, _ = orp.encode_quantize_global(rp, ci, a, bits, seed, t, G, d=d)
+        s, B = orp.expand_global_scales(s0, d), 512
+    _, beta = orp.decode(d, bits, B, w, mask, c, s, lr=lr, beta=beta, want_ghat=False)
+    return beta
+
+
 def oracle_sample_rate(wl, code, bits, bucket, target_s=12.0):
     """Time the CPU oracle (as it stands, one thread) on a bounded sample of the workload:
     whole pack blocks through encode + quantise + pack + decode + update."""
@@ -123,8 +138,7 @@ def oracle_sample_rate(wl, code, bits, bucket, target_s=12.0):
 
     def run(dd):
         t0 = time.perf_counter()
-        c, s, _, _ = orp.encode_quantize(rp, ci, a, bits, bucket, wl.seed, 0, G[:, :dd], d=dd)
-        orp.decode(dd, bits, bucket, w, mask, c, s, lr=lr, beta=beta[:dd], want_ghat=False)
+        oracle_round(orp, code, bits, bucket, wl.seed, 0, G[:, :dd], dd, mask, lr, beta[:dd])
         return time.perf_counter() - t0
 
     t_small = run(d_s)
@@ -137,15 +151,19 @@ def oracle_sample_rate(wl, code, bits, bucket, target_s=12.0):
 
 
 def build_code(agc, wl, bucket):
+    """Bits (from the allocator where the workload says so) and code weights. With the global
+    norm (bucket 0) the variance dimension of the design is kept at 512, so that the bucket-wise
+    and the global-norm runs encode with the same bits and weights."""
     from synth import configs as cfgs
+    phi_dim = float(bucket) if bucket else 512.0
     if wl.bits is None:
-        bits, _ = agc.agc_bit_allocate(wl.p, wl.z_tot, b_min=2, b_max=wl.bits_range[1], phi_dim=float(bucket))
+        bits, _ = agc.agc_bit_allocate(wl.p, wl.z_tot, b_min=2, b_max=wl.bits_range[1], phi_dim=phi_dim)
     else:
         bits = wl.bits
     sup = cfgs.cyclic_support(wl)
     srp = np.arange(0, wl.n * wl.s + 1, wl.s, dtype=np.int32)
     sci = np.array(sum(sup, []), np.int32)
-    rp, ci, a, w, _ = agc.agc_code_build(wl.n, wl.k, wl.p, bits, float(bucket), mode=agc.AGC_CODE_SUPPORT,
+    rp, ci, a, w, _ = agc.agc_code_build(wl.n, wl.k, wl.p, bits, phi_dim, mode=agc.AGC_CODE_SUPPORT,
                                          sup_row_ptr=srp, sup_col_idx=sci)
     return (rp, ci, a, w), np.asarray(bits, np.uint8)
 
@@ -170,8 +188,7 @@ def run_reference(args, wl, bucket):
     times = []
     for t in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        c, s, _, _ = orp.encode_quantize(rp, ci, a, bits, bucket, wl.seed, t, G, d=d_s)
-        _, beta = orp.decode(d_s, bits, bucket, w, masks[t], c, s, lr=lr, beta=beta, want_ghat=False)
+        beta = oracle_round(orp, code, bits, bucket, wl.seed, t, G, d_s, masks[t], lr, beta)
         if t >= args.warmup:
             times.append(time.perf_counter() - t0)
     tot = sum(times)
@@ -201,7 +218,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
-    ap.add_argument("--bucket", type=int, default=512)
+    ap.add_argument("--bucket", type=int, default=512, help="128, 256, 512, or 0 = one norm per worker (two-pass encode)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -292,7 +309,7 @@ def main():
     # the two-track decode + Adam step (Sec. V-E) on the same messages: timed apart, not part of the step
     tt_ms = None
     if R == 1 and not args.no_two_track:
-        v2 = agc.agc_two_track_vector(wl.n, wl.k, wl.p, bits, float(bucket), rp, a)
+        v2 = agc.agc_two_track_vector(wl.n, wl.k, wl.p, bits, float(bucket) if bucket else 512.0, rp, a)
         m_t = torch.zeros(wl.d, dtype=torch.float32, device=dev)
         u_t = torch.zeros(wl.d, dtype=torch.float32, device=dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -80,7 +80,10 @@ typedef struct agc_plan agc_plan_t;
  *   w          host, n entries: decoding coefficients w_i
  *   p          host, n entries: straggler probabilities, 0 <= p_i < 1
  *   bits       host, n entries: b_i in 2..8 (1 with AGC_FLAG_ALLOW_1BIT)
- *   bucket     coordinates per scale: 128, 256 or 512
+ *   bucket     coordinates per scale: 128, 256 or 512; 0 = ONE l2 norm per worker over all d
+ *              coordinates, the main formulation of Sec. II-B (the encoder then reads the
+ *              partial gradients twice: block sums of squares, their pairwise-tree
+ *              reduction, rounding with the global norm; scales holds n entries)
  *   seed       key of the counter-based random stream of the stochastic rounding
  *   flags      AGC_FLAG_*
  * All host arrays are copied. Unless AGC_FLAG_NO_UNBIASED_CHECK is set the
@@ -98,7 +101,8 @@ void agc_plan_destroy(agc_plan_t *plan);
 /* Bytes of the concatenated messages: sum_i 4 * 16 * b_i * ceil(d/512)
  * (payload of Sec. II-B: z_i bits per coordinate, padded to whole blocks). */
 size_t agc_codes_bytes(const agc_plan_t *plan);
-/* Bytes of the scales array: 4 * n * ceil(d / bucket) (the norms of Eq. quant_def). */
+/* Bytes of the scales array: 4 * n * ceil(d / bucket) (the norms of Eq. quant_def);
+ * 4 * n with the global norm (bucket 0). */
 size_t agc_scales_bytes(const agc_plan_t *plan);
 /* Byte offset of worker i's message inside the codes buffer (multiple of 64);
  * i = n gives agc_codes_bytes. Returns (size_t)-1 for a bad index. */

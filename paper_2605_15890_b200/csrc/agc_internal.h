@@ -71,6 +71,8 @@ struct AgcEncParams {
     const int32_t *grp_wk_ptr;   // n_groups+1
     const int32_t *grp_workers;  // workers of each group
     const float *G;
+    float *partials;             // global norm: n x nblk block sums of squares
+    const float *ginv;           // global norm: n reciprocal scales (0 = flushed worker)
     uint32_t *codes;
     float *scales;
     uint32_t *status;
@@ -95,6 +97,7 @@ struct AgcDecParams {
     long long d, nblk, nb;
     int n, R;
     int rows_per_bucket;
+    int global_norm = 0;    // one scale per worker: scales[i]
     float lr0;              // learning rate of the single realisation (R == 1)
     const float *lr;        // device, R learning rates (per-realisation mode with beta)
     uint32_t *status = nullptr;  // AGC_STATUS_* bits are OR-ed into it (ring kernel), may be NULL
@@ -113,6 +116,8 @@ struct agc_plan {
     int bucket = 0;
     uint64_t seed = 0;
     long long first_block = 0;
+    bool global_norm = false;     // one l2 norm per worker (bucket argument 0)
+    float *d_partials = nullptr, *d_chunk_sums = nullptr, *d_ginv = nullptr;
     uint32_t flags = 0;
     int device = 0, sm_count = 0;
     std::vector<int32_t> row_ptr, col_idx;

@@ -90,6 +90,7 @@ void free_device(agc_plan *p)
     cudaFree(p->d_bits); cudaFree(p->d_wdesc); cudaFree(p->d_edesc); cudaFree(p->d_word_off);
     cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_op_ptr); cudaFree(p->d_ops); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
     cudaFree(p->d_weff); cudaFree(p->d_lr); cudaFree(p->d_v);
+    cudaFree(p->d_partials); cudaFree(p->d_chunk_sums); cudaFree(p->d_ginv);
     cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
     cudaFree(p->h_mask); cudaFree(p->h_status);
 }
@@ -105,7 +106,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     *out = nullptr;
     if (n_workers < 1 || k_parts < 1 || d < 1 || d > (int64_t(1) << 31) - 1024) return AGC_ERR_ARG;
     if (!row_ptr || !col_idx || !a || !w || !p || !bits) return AGC_ERR_ARG;
-    if (bucket != 128 && bucket != 256 && bucket != 512) return AGC_ERR_ARG;
+    if (bucket != 0 && bucket != 128 && bucket != 256 && bucket != 512) return AGC_ERR_ARG;
     if (row_ptr[0] != 0) return AGC_ERR_ARG;
     for (int i = 0; i < n_workers; ++i) {
         if (row_ptr[i + 1] < row_ptr[i]) return AGC_ERR_ARG;
@@ -135,11 +136,12 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     pl->n = n_workers;
     pl->k = k_parts;
     pl->d = d;
-    pl->bucket = int(bucket);
+    pl->global_norm = bucket == 0;
+    pl->bucket = bucket ? int(bucket) : AGC_BLOCK;   // the global norm runs the 512-block kernels
     pl->seed = seed;
     pl->flags = flags;
     pl->nblk = (d + AGC_BLOCK - 1) / AGC_BLOCK;
-    pl->nb = (d + bucket - 1) / bucket;
+    pl->nb = bucket ? (d + bucket - 1) / bucket : 1;
     pl->row_ptr.assign(row_ptr, row_ptr + n_workers + 1);
     pl->col_idx.assign(col_idx, col_idx + nnz);
     pl->a.assign(a, a + nnz);
@@ -214,6 +216,13 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc) rc = upload(&pl->d_grp_wk_ptr, grp_wk_ptr);
     if (!rc) rc = upload(&pl->d_grp_workers, grp_workers);
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
+    if (!rc && pl->global_norm) {
+        const size_t nchunk = size_t((pl->nblk + 1023) / 1024);
+        if (cudaMalloc(reinterpret_cast<void **>(&pl->d_partials), sizeof(float) * size_t(n_workers) * size_t(pl->nblk)) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void **>(&pl->d_chunk_sums), sizeof(float) * size_t(n_workers) * nchunk) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void **>(&pl->d_ginv), sizeof(float) * n_workers) != cudaSuccess)
+            rc = AGC_ERR_NOMEM;
+    }
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_v), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_lr), sizeof(float) * AGC_MAX_R) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc) rc = agc_encode_prepare(pl);

@@ -58,5 +58,5 @@ class Session:
         return self.codes.cpu().numpy().view(np.uint32)
 
     def scales_host(self):
-        nb = (self.d + self.bucket - 1) // self.bucket
+        nb = (self.d + self.bucket - 1) // self.bucket if self.bucket else 1
         return self.scales.cpu().numpy().reshape(self.n, nb)

@@ -435,3 +435,45 @@ def test_two_track_decode_and_adam_steps(agc, torch, B, d):
         assert (beta.cpu().numpy().view(np.uint32) == ob.view(np.uint32)).all()
     assert int(ses.status.item()) == 0
     ses.close()
+
+
+@pytest.mark.parametrize("d,direct", [(300, False), (5000, False), (5000, True), (600_001, False)])
+def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
+    """The paper's main formulation (one l2 norm per worker, bucket = 0): two-pass encode
+    against the oracle's global-norm encoder, bit for bit, then decode and fused update. The
+    largest case spans several 1024-block chunks of the norm reduction; one worker is zero."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(d)
+    n = k = 6
+    bits = np.array([1, 2, 3, 4, 6, 8], np.uint8)
+    p = rng.uniform(0.05, 0.4, n)
+    rp, ci, a, w = _codes.identity_code(n)
+    w = (1.0 / (1.0 - p)).astype(np.float32)
+    G_host = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 2, (k, 1))).astype(np.float32)
+    G_host[3] = 0.0
+    flags = agc.AGC_FLAG_ALLOW_1BIT | (agc.AGC_FLAG_FORCE_DIRECT if direct else 0)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=0, seed=17, flags=flags)
+    ld = (d + 3) // 4 * 4
+    G = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+    G[:, :d] = torch.from_numpy(G_host)
+    ses.codes.fill_(-1)
+    ses.scales.fill_(-1.0)
+    mask = np.array([1, 1, 0, 1, 1, 1], np.uint8)
+    lr = np.array([0.01], np.float32)
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    beta = torch.from_numpy(beta0.copy()).cuda()
+    ghat = torch.empty((1, d), dtype=torch.float32, device="cuda")
+    for rnd in (0, 1):
+        ses.encode(G, rnd)
+    ses.decode(torch.from_numpy(mask).cuda(), lr=lr, ghat=ghat, beta=beta)
+    torch.cuda.synchronize()
+    assert int(ses.status.item()) == 0 and ses.uses_tma == (not direct)
+    oc, osc, st, _ = orp.encode_quantize_global(rp, ci, a, bits, 17, 1, G_host)
+    assert st == 0 and osc[3] == 0.0
+    assert (ses.scales_host()[:, 0].view(np.uint32) == osc.view(np.uint32)).all()
+    bad = np.nonzero(ses.codes_host() != oc)[0]
+    assert bad.size == 0, f"{bad.size} code words differ, first at {bad[:5]}"
+    og, ob = orp.decode(d, bits, 512, w, mask[None], oc, orp.expand_global_scales(osc, d), lr=lr, beta=beta0)
+    assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
+    assert (beta.cpu().numpy().view(np.uint32) == ob.view(np.uint32)).all()
+    ses.close()
