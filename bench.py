@@ -29,7 +29,7 @@ UNIT = "coords/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the encode kernel, from the ncu
 # capture summarised under profiles/ (bytes per coordinate of the captured case, scaled to d).
-NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 142.28}   # profiles/k1_encode_staged_cfg3_d4M.md
+NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 142.28}   # bucket-wise encoder, bucket 512
 
 
 def workload(name):
@@ -348,7 +348,7 @@ def main():
         peak, which = measured_hbm_peak()
         k1_bytes = k1_algorithmic_bytes(wl, bits, bucket)
         achieved = k1_bytes / (k1_ms * 1e-3) / 1e9
-        tpc = NCU_TRAFFIC_BYTES_PER_COORD.get(wl.name)
+        tpc = NCU_TRAFFIC_BYTES_PER_COORD.get(wl.name) if bucket == 512 else None
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
