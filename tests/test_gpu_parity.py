@@ -477,3 +477,46 @@ def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
     assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
     assert (beta.cpu().numpy().view(np.uint32) == ob.view(np.uint32)).all()
     ses.close()
+
+
+def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch):
+    """Lemma 1 as a measured experiment: 20 rounds x 64 straggler realisations through the CUDA
+    path (fresh rounding each round, fresh Bernoulli masks each realisation). The mean of
+    g_hat approaches sum_j g_j (unbiasedness, Eq. exp_g2_quant) and the mean squared error
+    stays below C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 with ||g_j||^2 = C."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(31)
+    n = k = 8
+    d, B = 4096, 512
+    bits = np.array([2, 3, 4, 6, 2, 5, 3, 4], np.uint8)
+    p = rng.uniform(0.05, 0.4, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B)
+    A = od.csr_to_dense(rp, ci, a.astype(np.float64), k)
+    G_host = rng.standard_normal((k, d)).astype(np.float32)
+    G_host /= np.linalg.norm(G_host.astype(np.float64), axis=1, keepdims=True).astype(np.float32)   # C = 1
+    g = G_host.astype(np.float64).sum(axis=0)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=77)
+    G = torch.from_numpy(G_host).cuda()
+    rounds, R = 20, 64
+    ghat = torch.empty((R, d), dtype=torch.float32, device="cuda")
+    mean = np.zeros(d)
+    mse = 0.0
+    for t in range(rounds):
+        masks = (rng.random((R, n)) >= p).astype(np.uint8)
+        ses.encode(G, t)
+        ses.decode(torch.from_numpy(masks).cuda(), ghat=ghat)
+        gh = ghat.cpu().numpy().astype(np.float64)
+        mean += gh.sum(axis=0)
+        mse += ((gh - g) ** 2).sum()
+    N = rounds * R
+    mean /= N
+    mse /= N
+    bound = od.lemma1_bound(A, w.astype(np.float64), p, bits, B, C=1.0)
+    assert mse <= bound * 1.05
+    assert mse >= 0.05 * bound                 # the experiment is not vacuous
+    # unbiasedness: the realisations of one round share their rounding noise, so the mean has
+    # at least `rounds` independent terms: its error is below 3 sqrt(mse / rounds) and far
+    # below the error of a single estimate
+    assert np.linalg.norm(mean - g) <= 3.0 * np.sqrt(mse / rounds)
+    assert np.linalg.norm(mean - g) <= 0.3 * np.sqrt(mse)
+    ses.close()
