@@ -106,9 +106,9 @@ def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
     assert out["tma"] == (not direct)
 
 
-@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups"])
+@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers"])
 def test_code_structures(agc, torch, kind):
-    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups"].index(kind))
+    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers"].index(kind))
     d = 3000
     if kind == "identity":
         n = k = 5
@@ -135,6 +135,11 @@ def test_code_structures(agc, torch, kind):
         bits = rng.integers(2, 9, n).astype(np.uint8)
         p = rng.uniform(0.05, 0.5, n)
         code = _codes.cyclic_code(p, bits, k, 40, 512)
+    elif kind == "many_workers":   # hundreds of workers: many groups in both kernels
+        n = k = 300
+        bits = rng.integers(1, 9, n).astype(np.uint8)
+        p = rng.uniform(0.01, 0.6, n)
+        code = _codes.cyclic_code(p, bits, k, 2, 512)
     else:                          # many worker groups per block in the staged kernel
         n = k = 100
         bits = rng.integers(1, 9, n).astype(np.uint8)
