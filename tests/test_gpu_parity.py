@@ -525,3 +525,47 @@ def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch):
     assert np.linalg.norm(mean - g) <= 3.0 * np.sqrt(mse / rounds)
     assert np.linalg.norm(mean - g) <= 0.3 * np.sqrt(mse)
     ses.close()
+
+
+@pytest.mark.parametrize("d,B", [(1, 128), (513, 256), (70_001, 512), (40_000, 0)])
+def test_kernels_write_nothing_outside_their_outputs(agc, torch, d, B):
+    """Guard words before and after every output buffer (messages, scales, g_hat, parameters,
+    Adam state) must survive encode, decode, the collapsed update and the two-track step."""
+    rng = np.random.default_rng(d + B)
+    n = k = 9
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B if B else 512)
+    plan = agc.agc_plan_create(n, k, d, rp, ci, a, w, p, bits, B, 3, agc.AGC_FLAG_ALLOW_1BIT)
+    pad = 1024                                             # floats / words of guard on each side
+    def guarded(nelem, dtype, fill):
+        buf = torch.full((nelem + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + nelem]
+    GUARD_I, GUARD_F = 0x5A5A5A5A, -12345.5
+    codes_all, codes = guarded(agc.agc_codes_bytes(plan) // 4, torch.int32, GUARD_I)
+    scales_all, scales = guarded(agc.agc_scales_bytes(plan) // 4, torch.float32, GUARD_F)
+    outs = {name: guarded(R_ * d, torch.float32, GUARD_F) for name, R_ in
+            [("ghat", 3), ("beta", 1), ("gw", 1), ("gv", 1), ("m", 1), ("u", 1)]}
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ld = (d + 3) // 4 * 4
+    G = torch.from_numpy(rng.standard_normal((k, ld)).astype(np.float32)).cuda()
+    masks = torch.from_numpy((rng.random((3, n)) > 0.3).astype(np.uint8)).cuda()
+    lr = np.array([1e-3, 2e-3, 3e-3], np.float32)
+    for name in ("beta", "m", "u"):
+        outs[name][1].zero_()
+    agc.agc_encode_quantize(plan, G, ld, 4, codes, scales, status)
+    agc.agc_decode(plan, codes, scales, masks, 3, lr, outs["ghat"][1], outs["beta"][1], status)
+    agc.agc_decode(plan, codes, scales, masks, 3, lr, None, outs["beta"][1], status)          # collapsed
+    agc.agc_decode_two_track(plan, codes, scales, masks[0], w, outs["gw"][1], outs["gv"][1], outs["beta"][1],
+                             outs["m"][1], outs["u"][1], adam=(1e-3, 0.9, 0.999, 1e-8, 1), status_dev=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    def check(all_, fill):
+        assert bool((all_[:pad] == fill).all()) and bool((all_[-pad:] == fill).all())
+    check(codes_all, GUARD_I)
+    check(scales_all, GUARD_F)
+    for name, (all_, inner) in outs.items():
+        check(all_, GUARD_F)
+        assert not bool((inner == GUARD_F).any()), name      # every output element was written
+    assert not bool((scales == GUARD_F).any())
+    agc.agc_plan_destroy(plan)
