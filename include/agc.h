@@ -315,6 +315,14 @@ int agc_code_build(int n, int k, const double *p, const uint8_t *bits, double ph
                    int32_t *col_out, float *a_out, float *w_out, double *Y_out);
 
 /*
+ * agc_eta_balance - the error-balance factor suggested in Sec. V-B:
+ * eta = mean(p) * 4 (2^(Z_tot/n - 1) - 1)^2 / phi_dim, which makes eta * phi(Z_tot / n) equal
+ * to the average straggler probability; pass it as `eta` to agc_bit_allocate,
+ * agc_code_build and agc_two_track_vector. Host only.
+ */
+int agc_eta_balance(int n, const double *p, int Z_tot, double phi_dim, double *eta_out);
+
+/*
  * agc_selftest_division - diagnostic. The encoder forms the reciprocal scale L_i 2^15 / S
  * of Eq. quant_def's normalisation with its own branch-free division; this call compares
  * it on the current device with the IEEE-754 correctly rounded quotient for every

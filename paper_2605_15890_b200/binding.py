@@ -83,6 +83,8 @@ def _load():
     L.agc_code_build.restype = C.c_int
     L.agc_selftest_division.argtypes = [C.POINTER(C.c_ulonglong)]
     L.agc_selftest_division.restype = C.c_int
+    L.agc_eta_balance.argtypes = [C.c_int, f64p, C.c_int, C.c_double, f64p]
+    L.agc_eta_balance.restype = C.c_int
     L.agc_strerror.argtypes = [C.c_int]
     L.agc_strerror.restype = C.c_char_p
     L.agc_version.argtypes = []
@@ -228,6 +230,13 @@ def agc_round_host(plan, G_host, ld_host, rnd, mask_host, ghat_host, stream=None
     _check(_lib.agc_round_host(plan, addr(G_host), ld_host, rnd, addr(mask_host), addr(ghat_host),
                                C.byref(st), _stream(stream)))
     return st.value
+
+
+def agc_eta_balance(p, z_tot, phi_dim):
+    p = _np(p, np.float64)
+    eta = C.c_double(0.0)
+    _check(_lib.agc_eta_balance(len(p), _hp(p, C.c_double), z_tot, phi_dim, C.byref(eta)))
+    return eta.value
 
 
 def agc_selftest_division():

@@ -364,3 +364,17 @@ extern "C" int agc_two_track_vector(int n, int k, const double *p, const uint8_t
     }
     return AGC_OK;
 }
+
+extern "C" int agc_eta_balance(int n, const double *p, int Z_tot, double phi_dim, double *eta_out)
+{
+    if (n < 1 || !p || !eta_out || !(phi_dim > 0.0) || Z_tot < 2 * n) return AGC_ERR_ARG;
+    double mean = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (!(p[i] >= 0.0 && p[i] < 1.0)) return AGC_ERR_PROB;
+        mean += p[i];
+    }
+    mean /= double(n);
+    const double lev = std::exp2(double(Z_tot) / double(n) - 1.0) - 1.0;
+    *eta_out = mean * 4.0 * lev * lev / phi_dim;
+    return AGC_OK;
+}

@@ -139,3 +139,19 @@ def test_two_track_vector_against_oracle():
             v = agc.agc_two_track_vector(n, k, p, bits, 256.0, rp, vals.astype(np.float32), lam=lam)
             want = od.two_track_decoder(A, p, bits, 256, lam=lam)
             assert np.allclose(v, want, rtol=2e-6, atol=0)
+
+
+def test_eta_balance_and_its_use_in_the_design_calls():
+    """Sec. V-B: the suggested eta against the oracle; with it the allocator and the code builder
+    of the library still agree with the oracle's (eta enters phi everywhere)."""
+    rng = np.random.default_rng(6)
+    n, k, dim, z_tot = 10, 10, 512, 40
+    p = rng.uniform(0.05, 0.5, n)
+    eta = agc.agc_eta_balance(p, z_tot, float(dim))
+    assert np.isclose(eta, od.eta_balance(p, z_tot, dim), rtol=1e-12)
+    assert np.isclose(eta * od.phi(z_tot // n, dim), p.mean(), rtol=1e-12)
+    bits, F = agc.agc_bit_allocate(p, z_tot, b_max=8, phi_dim=float(dim), eta=eta)
+    obits, oF = od.bit_allocate_low_complexity(p, z_tot, dim, b_max=8, eta=eta)
+    assert bits.sum() == z_tot and np.isclose(F, oF, rtol=1e-9)
+    rp, ci, a, w, Y = agc.agc_code_build(n, k, p, bits, float(dim), eta=eta)
+    assert np.allclose(Y, od.optimal_row_sums(p, bits, k, dim, eta=eta), rtol=1e-9)
