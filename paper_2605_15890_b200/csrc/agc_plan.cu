@@ -68,17 +68,39 @@ bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::ve
         *max_rows = std::max<int>(*max_rows, int(cur_rows.size()));
         cur_rows.clear();
     };
-    for (int i = 0; i < pl.n; ++i) {
-        const int e0 = pl.row_ptr[i], e1 = pl.row_ptr[i + 1];
-        if (e1 - e0 > AGC_MAX_STAGE_ROWS) return false;
+    for (int i = 0; i < pl.n; ++i)
+        if (pl.row_ptr[i + 1] - pl.row_ptr[i] > AGC_MAX_STAGE_ROWS) return false;
+    // The order of the tasks is free (a task's output place depends on its worker only), so a
+    // group is filled with the workers that bring the fewest new partition rows: banded and
+    // cyclic supports come out in their natural order, scattered supports are clustered and
+    // their rows are staged fewer times. Ties go to the lowest index.
+    std::vector<char> taken(pl.n, 0);
+    auto fresh_rows = [&](int i) {
         int fresh = 0;
-        for (int e = e0; e < e1; ++e) fresh += !in_group[pl.col_idx[e]];
-        if (int(cur_rows.size()) + fresh > AGC_MAX_STAGE_ROWS) flush();
-        for (int e = e0; e < e1; ++e) {
+        for (int e = pl.row_ptr[i]; e < pl.row_ptr[i + 1]; ++e) fresh += !in_group[pl.col_idx[e]];
+        return fresh;
+    };
+    int first_free = 0;
+    for (int placed = 0; placed < pl.n; ++placed) {
+        while (taken[first_free]) ++first_free;
+        int best = first_free, best_fresh = fresh_rows(first_free);
+        if (!cur_rows.empty() && pl.n <= 4096) {
+            for (int i = first_free + 1; i < pl.n && best_fresh > 0; ++i) {
+                if (taken[i]) continue;
+                const int f = fresh_rows(i);
+                if (f < best_fresh) { best = i; best_fresh = f; }
+            }
+        }
+        if (int(cur_rows.size()) + best_fresh > AGC_MAX_STAGE_ROWS) {
+            flush();
+            best = first_free;          // a new group starts from the lowest free worker
+        }
+        for (int e = pl.row_ptr[best]; e < pl.row_ptr[best + 1]; ++e) {
             const int j = pl.col_idx[e];
             if (!in_group[j]) { in_group[j] = 1; cur_rows.push_back(j); }
         }
-        grp_workers.push_back(i);
+        grp_workers.push_back(best);
+        taken[best] = 1;
     }
     flush();
     return true;

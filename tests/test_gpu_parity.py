@@ -106,9 +106,9 @@ def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
     assert out["tma"] == (not direct)
 
 
-@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers"])
+@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered"])
 def test_code_structures(agc, torch, kind):
-    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers"].index(kind))
+    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered"].index(kind))
     d = 3000
     if kind == "identity":
         n = k = 5
@@ -135,6 +135,18 @@ def test_code_structures(agc, torch, kind):
         bits = rng.integers(2, 9, n).astype(np.uint8)
         p = rng.uniform(0.05, 0.5, n)
         code = _codes.cyclic_code(p, bits, k, 40, 512)
+    elif kind == "scattered":      # supports scattered over the partitions (not banded): clustered groups
+        n, k = 60, 90
+        bits = rng.integers(1, 9, n).astype(np.uint8)
+        p = rng.uniform(0.01, 0.5, n)
+        alpha = np.zeros((n, k))
+        for j in range(k):
+            holders = rng.choice(n, size=3, replace=False)
+            alpha[holders, j] = rng.uniform(0.2, 1.0, 3)
+        alpha /= alpha.sum(0, keepdims=True)
+        rp_, ci_, vals_ = od.alpha_to_csr(alpha)
+        _, w_ = od.physical_coefficients(alpha, p)
+        code = (rp_, ci_, vals_.astype(np.float32), w_.astype(np.float32))
     elif kind == "many_workers":   # hundreds of workers: many groups in both kernels
         n = k = 300
         bits = rng.integers(1, 9, n).astype(np.uint8)
@@ -150,6 +162,7 @@ def test_code_structures(agc, torch, kind):
     out, ref = run_both(agc, torch, G, code, p, bits, 512, 77, 3, masks)
     assert_exact(out, ref)
     assert out["tma"] == (kind != "wide_rows")
+    assert G.shape[0] == k
 
 
 def test_straggler_extremes_and_batched_decode(agc, torch):
