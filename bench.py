@@ -30,6 +30,10 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the encode kernel, from the ncu
 # capture summarised under profiles/ (bytes per coordinate of the captured case, scaled to d).
 NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 142.28}   # bucket-wise encoder, bucket 512
+# smsp__inst_executed.sum per (worker, pack block) task of the encode kernel from the same capture:
+# the kernel is bound by instruction issue, so the line also reports the issue rate it reaches
+# against 4 schedulers x 148 SMs x the SM clock sampled during the run.
+NCU_WARP_INST_PER_TASK = {"cfg3": 383.0}
 
 
 def workload(name):
@@ -64,6 +68,19 @@ def k2_algorithmic_bytes(wl, bits, bucket, masks_all, p):
     used = m.any(axis=1)                              # rounds x n
     per_worker = np.array([64 * int(b) * nblk + 4 * nb for b in bits], np.float64)
     return float((used * per_worker[None, :]).sum(axis=1).mean()) + 8.0 * wl.d
+
+
+def issue_rate(wl, bucket, k1_ms, clocks):
+    """Second ceiling of the encode kernel: warp instructions issued per second against the
+    issue capacity at the sampled SM clock (None where no instruction count was captured)."""
+    ipt = NCU_WARP_INST_PER_TASK.get(wl.name) if bucket == 512 else None
+    if ipt is None or not clocks or not clocks.get("sm_mhz"):
+        return None
+    tasks = wl.n * ((wl.d + 511) // 512)
+    achieved = ipt * tasks / (k1_ms * 1e-3)
+    peak = 148 * 4 * clocks["sm_mhz"] * 1e6
+    return {"bound": "alu", "achieved": achieved / 1e9, "peak": peak / 1e9, "unit": "G warp-inst/s",
+            "frac": achieved / peak, "warp_inst_per_task": ipt}
 
 
 class ClockSampler:
@@ -360,7 +377,8 @@ def main():
                              "achieved": achieved, "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
                              "frac": achieved / peak, "frac_of_8000": achieved / 8000.0,
                              "algorithmic_bytes": k1_bytes,
-                             "traffic": None if tpc is None else tpc * wl.d},
+                             "traffic": None if tpc is None else tpc * wl.d,
+                             "issue": issue_rate(wl, bucket, k1_ms, clocks)},
                 "clocks": clocks, "e2e": e2e,
                 "gpu_launches": args.steps * (2 + (1 if R > 1 else 0))}
         if not args.no_cpu_baseline:
