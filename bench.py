@@ -343,7 +343,9 @@ def main():
 
     # end to end through the host-buffer entry point (pinned host memory, copies timed)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and in_bytes > 16e9:
+        e2e = {"value": None, "unit": UNIT, "skipped": "host staging of %.0f GB of partial gradients not attempted" % (in_bytes / 1e9)}
+    elif not args.no_e2e:
         Gh = torch.empty((wl.k, wl.d), dtype=torch.float32).pin_memory()
         Gh.copy_(G[:, :wl.d])
         mh = masks_all[0, 0].cpu().pin_memory()
