@@ -196,16 +196,18 @@ def run_reference(args, wl, bucket):
     code, bits = build_code(agc, wl, bucket)
     rp, ci, a, w = code
     rate0, _, _ = oracle_sample_rate(wl, code, bits, bucket, target_s=2.0)
-    blocks = int(max(8, min(1 << 15, rate0 * 4.0 / 512)))   # about 4 s per step
+    # the whole run (warm-up + timed steps) is sized to about two minutes of host time
+    per_step_s = min(4.0, 120.0 / max(1, args.steps + args.warmup))
+    blocks = int(max(8, min(1 << 15, rate0 * per_step_s / 512)))
     d_s = blocks * 512
     G = cfgs.partials_numpy(wl, 0, d=d_s)
-    masks = cfgs.straggler_masks(wl, rounds=args.steps + args.warmup, realizations=1)
+    masks = cfgs.straggler_masks(wl, rounds=min(args.steps + args.warmup, 64), realizations=1)
     beta = np.zeros(d_s, np.float32)
     lr = np.array([1e-3], np.float32)
     times = []
     for t in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        beta = oracle_round(orp, code, bits, bucket, wl.seed, t, G, d_s, masks[t], lr, beta)
+        beta = oracle_round(orp, code, bits, bucket, wl.seed, t, G, d_s, masks[t % len(masks)], lr, beta)
         if t >= args.warmup:
             times.append(time.perf_counter() - t0)
     tot = sum(times)
