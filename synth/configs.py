@@ -68,6 +68,13 @@ def config5(seed=5, d=100_000_000):
                     bits=r.integers(1, 9, 100).astype(np.uint8), realizations=64)
 
 
+def shifted_exponential_probs(n, seed=0, psi_range=(0.1, 2.0), tau_th=1.1):
+    """Straggler probabilities of the paper's delay model (Sec. V-A / VI): worker i has rate
+    psi_i ~ U(psi_range) and misses the deadline tau_th with p_i = exp(-psi_i (tau_th - 1))."""
+    psi = _rng(seed, 21).uniform(psi_range[0], psi_range[1], n)
+    return np.exp(-psi * (tau_th - 1.0))
+
+
 def cyclic_support(wl):
     """Column lists of the cyclic assignment (sorted ascending)."""
     return [sorted(((i + t) % wl.k) for t in range(wl.s)) for i in range(wl.n)]

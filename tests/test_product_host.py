@@ -155,3 +155,22 @@ def test_eta_balance_and_its_use_in_the_design_calls():
     assert bits.sum() == z_tot and np.isclose(F, oF, rtol=1e-9)
     rp, ci, a, w, Y = agc.agc_code_build(n, k, p, bits, float(dim), eta=eta)
     assert np.allclose(Y, od.optimal_row_sums(p, bits, k, dim, eta=eta), rtol=1e-9)
+
+
+@pytest.mark.parametrize("n", [10, 50])
+def test_allocator_under_the_papers_delay_model(n):
+    """The setting of the paper's allocator figure: p_i from the shifted-exponential delay model
+    (psi ~ U(0.1, 2), deadline 1.1), residual budgets n and 5n. The library's Algorithm 1 stays
+    within 1 % of its own exact DP and never below the equal split."""
+    from synth import configs as cfgs
+    p = np.minimum(cfgs.shifted_exponential_probs(n, seed=n), 0.95)
+    for zres in (n, 5 * n):
+        bits, F = agc.agc_bit_allocate(p, 2 * n + zres, b_max=0, phi_dim=512.0)
+        _, F_dp = agc.agc_bit_allocate_dp(p, 2 * n + zres, b_max=0, phi_dim=512.0)
+        assert bits.sum() == 2 * n + zres and (bits >= 2).all()
+        assert F_dp * (1 + 1e-12) >= F >= 0.99 * F_dp
+        base, rem = divmod(zres, n)
+        order = np.argsort(p, kind="stable")
+        r_eq = np.zeros(n, int)
+        r_eq[order] = base + (np.arange(n) < rem)
+        assert F >= od.allocation_value(p, r_eq, 512) * (1 - 1e-12)
