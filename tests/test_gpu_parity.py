@@ -582,3 +582,60 @@ def test_kernels_write_nothing_outside_their_outputs(agc, torch, d, B):
         assert not bool((inner == GUARD_F).any()), name      # every output element was written
     assert not bool((scales == GUARD_F).any())
     agc.agc_plan_destroy(plan)
+
+
+def test_config5_full_size_sampled_blocks(agc, torch):
+    """cfg5 at its full size (n = k = 100, s = 5, d = 10^8 Student-t(3) values, bits 1..8, 64
+    straggler realisations per encode, 40 GB of partial gradients, messages beyond 4 GiB):
+    sampled pack blocks - first, last, around the 4 GiB byte offset of the message buffer,
+    random ones - are recomputed by the oracle from the same inputs. Codes and scales bit for
+    bit; the collapsed 64-realisation update within 1e-5 of the sequential definition."""
+    from paper_2605_15890_b200.session import Session
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs about 50 GB of device memory")
+    wl = cfgs.config5()
+    B = 512
+    rp, ci, a, w = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, B)
+    ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, wl.bits, bucket=B, seed=wl.seed, flags=agc.AGC_FLAG_ALLOW_1BIT)
+    G = cfgs.partials_torch(wl, "cuda:0", ld=wl.d)
+    masks = cfgs.straggler_masks(wl, rounds=1)[0]                      # 64 x 100
+    lr = np.full(wl.realizations, 1e-3, np.float32)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    beta0 = torch.empty(wl.d, dtype=torch.float32, device="cuda").normal_(generator=gen)
+    beta = beta0.clone()
+    ses.encode(G, 3)
+    ses.decode(torch.from_numpy(masks).cuda(), lr=lr, beta=beta)
+    torch.cuda.synchronize()
+    assert int(ses.status.item()) & 4 == 0
+    nblk = (wl.d + 511) // 512
+    off = orp.worker_word_offsets(wl.d, wl.bits)
+    assert int(off[-1]) * 4 > (1 << 32)
+    # blocks whose words straddle the 4 GiB byte offset for some worker
+    cross = int(np.searchsorted(off * 4, 1 << 32) - 1)
+    q_cross = int(((1 << 32) // 4 - int(off[cross])) // (16 * int(wl.bits[cross])))
+    rng = np.random.default_rng(9)
+    sample = {0, 1, nblk - 2, nblk - 1, max(0, q_cross - 1), min(nblk - 1, q_cross), min(nblk - 1, q_cross + 1)} | \
+        {int(x) for x in rng.integers(0, nblk, 40)}
+    for q in sorted(sample):
+        m0, m1 = q * 512, min((q + 1) * 512, wl.d)
+        blk = np.zeros((wl.k, 512), np.float32)
+        blk[:, :m1 - m0] = G[:, m0:m1].cpu().numpy()
+        oc, osc, st, _ = orp.encode_block(rp, ci, a, wl.bits, B, wl.seed, 3, q, blk)
+        wb = 0
+        for i in range(wl.n):
+            b = int(wl.bits[i])
+            lo = int(off[i]) + q * 16 * b
+            got = ses.codes[lo:lo + 16 * b].cpu().numpy().view(np.uint32)
+            assert (got == oc[wb:wb + 16 * b]).all(), (q, i)
+            wb += 16 * b
+        got_s = ses.scales.view(wl.n, -1)[:, q].cpu().numpy()
+        assert (got_s.view(np.uint32) == osc[:, 0].view(np.uint32)).all(), q
+        want = beta0[m0:m1].cpu().numpy().astype(np.float32)
+        for r in range(wl.realizations):
+            og = orp.decode_block(wl.bits, B, w, masks[r], oc, osc)
+            want = (want.astype(np.float64) - np.float64(lr[r]) * og[:m1 - m0].astype(np.float64)).astype(np.float32)
+        got_b = beta[m0:m1].cpu().numpy()
+        assert np.abs(got_b - want).max() <= 1e-5 * max(1.0, np.abs(want).max()), q
+    ses.close()
