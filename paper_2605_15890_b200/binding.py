@@ -62,6 +62,8 @@ def _load():
     L.agc_plan_uses_tma.restype = C.c_int
     L.agc_encode_quantize.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, vp, vp]
     L.agc_encode_quantize.restype = C.c_int
+    L.agc_encode_quantize_rows.argtypes = [vp, vp, C.c_uint64, vp, vp, vp, vp]
+    L.agc_encode_quantize_rows.restype = C.c_int
     L.agc_decode.argtypes = [vp, vp, vp, vp, C.c_int, f32p, vp, vp, vp, vp]
     L.agc_decode.restype = C.c_int
     L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
@@ -175,6 +177,12 @@ def agc_plan_uses_tma(plan):
 def agc_encode_quantize(plan, G_dev, ld, rnd, codes_dev, scales_dev, status_dev=None, stream=None):
     _check(_lib.agc_encode_quantize(plan, _dev(G_dev), ld, rnd, _dev(codes_dev), _dev(scales_dev),
                                     _dev(status_dev), _stream(stream)))
+
+
+def agc_encode_quantize_rows(plan, G_rows_dev, rnd, codes_dev, scales_dev, status_dev=None, stream=None):
+    """G_rows_dev: device array of k row addresses (a torch int64 CUDA tensor)."""
+    _check(_lib.agc_encode_quantize_rows(plan, _dev(G_rows_dev), rnd, _dev(codes_dev), _dev(scales_dev),
+                                         _dev(status_dev), _stream(stream)))
 
 
 def agc_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host=None, ghat_dev=None, beta_dev=None,

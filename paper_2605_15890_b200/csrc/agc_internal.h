@@ -71,6 +71,7 @@ struct AgcEncParams {
     const int32_t *grp_wk_ptr;   // n_groups+1
     const int32_t *grp_workers;  // workers of each group
     const float *G;
+    const float *const *G_rows;  // k row pointers instead of G (direct kernel only), or NULL
     float *partials;             // global norm: n x nblk block sums of squares
     const float *ginv;           // global norm: n reciprocal scales (0 = flushed worker)
     uint32_t *codes;
@@ -155,8 +156,8 @@ struct agc_plan {
     void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled entry point
 };
 
-int agc_launch_encode(agc_plan *plan, const float *G, long long ld, uint64_t round, void *codes,
-                      float *scales, uint32_t *status, cudaStream_t stream);
+int agc_launch_encode(agc_plan *plan, const float *G, const float *const *G_rows, long long ld, uint64_t round,
+                      void *codes, float *scales, uint32_t *status, cudaStream_t stream);
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
                       int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
                       cudaStream_t stream);

@@ -288,7 +288,19 @@ extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t
     if ((ld & 3) || (reinterpret_cast<uintptr_t>(G_dev) & 15) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
         (reinterpret_cast<uintptr_t>(scales_dev) & 3))
         return AGC_ERR_ALIGN;
-    return agc_launch_encode(plan, G_dev, ld, round, codes_dev, scales_dev, status_dev,
+    return agc_launch_encode(plan, G_dev, nullptr, ld, round, codes_dev, scales_dev, status_dev,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int agc_encode_quantize_rows(agc_plan_t *plan, const float *const *G_rows_dev, uint64_t round,
+                                        void *codes_dev, float *scales_dev, uint32_t *status_dev,
+                                        void *cuda_stream)
+{
+    if (!plan || !G_rows_dev || !codes_dev || !scales_dev) return AGC_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(G_rows_dev) & 7) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
+        (reinterpret_cast<uintptr_t>(scales_dev) & 3))
+        return AGC_ERR_ALIGN;
+    return agc_launch_encode(plan, nullptr, G_rows_dev, 0, round, codes_dev, scales_dev, status_dev,
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -345,7 +357,7 @@ extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_
         cudaMemcpyAsync(plan->h_mask, mask_host, plan->n, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemsetAsync(plan->h_status, 0, sizeof(uint32_t), st) != cudaSuccess)
         return AGC_ERR_CUDA;
-    int rc = agc_launch_encode(plan, plan->h_G, ld_dev, round, plan->h_codes, plan->h_scales, plan->h_status, st);
+    int rc = agc_launch_encode(plan, plan->h_G, nullptr, ld_dev, round, plan->h_codes, plan->h_scales, plan->h_status, st);
     if (rc) return rc;
     rc = agc_launch_decode(plan, plan->h_codes, plan->h_scales, plan->h_mask, 1, nullptr, plan->h_ghat, nullptr,
                            plan->h_status, st);

@@ -639,3 +639,30 @@ def test_config5_full_size_sampled_blocks(agc, torch):
         got_b = beta[m0:m1].cpu().numpy()
         assert np.abs(got_b - want).max() <= 1e-5 * max(1.0, np.abs(want).max()), q
     ses.close()
+
+
+@pytest.mark.parametrize("B", [0, 256])
+def test_encode_from_separate_row_buffers(agc, torch, B):
+    """Partial gradients in k separate device buffers (an array of row pointers): the messages
+    must be those of the contiguous call, bit for bit."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(44)
+    n = k = 7
+    d = 9000
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.5, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B if B else 512)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=8, flags=agc.AGC_FLAG_ALLOW_1BIT)
+    G_host = rng.standard_normal((k, d)).astype(np.float32)
+    G = torch.from_numpy(G_host).cuda()
+    ses.encode(G, 6)
+    want_codes, want_scales = ses.codes.clone(), ses.scales.clone()
+    rows = [torch.from_numpy(G_host[j].copy()).cuda() for j in reversed(range(k))][::-1]   # separate allocations
+    ptrs = torch.tensor([r.data_ptr() for r in rows], dtype=torch.int64, device="cuda")
+    ses.codes.fill_(-1)
+    ses.scales.fill_(-1.0)
+    agc.agc_encode_quantize_rows(ses.plan, ptrs, 6, ses.codes, ses.scales, ses.status)
+    torch.cuda.synchronize()
+    assert bool((ses.codes == want_codes).all()) and bool((ses.scales.view(torch.int32) == want_scales.view(torch.int32)).all())
+    assert int(ses.status.item()) == 0
+    ses.close()
