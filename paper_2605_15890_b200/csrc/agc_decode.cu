@@ -5,6 +5,14 @@
 // One warp owns one 512-coordinate pack block. Lane l holds the 16 coordinates
 // {128c + 4l + e}, i.e. stream positions 16l..16l+15 of every worker's message, so it
 // reads 16*b_i contiguous bits per worker and never needs another lane's data.
+//
+// Kernels in this file:
+//   agc_decode_ring_kernel  persistent CTAs; a producer warp brings the received workers'
+//       words into a shared-memory ring with bulk copies, the consumer warps unpack them
+//       (one realisation, the collapsed multi-realisation update, or the two-track decode
+//       of Sec. V-E with the Adam step);
+//   agc_decode_kernel       the same arithmetic with plain global loads, for plans the
+//       ring cannot serve and for the allocation-free entry point at the end of the file.
 #include <cmath>
 #include <mutex>
 
