@@ -154,6 +154,10 @@ struct agc_plan {
     uint8_t *h_mask = nullptr;
     uint32_t *h_status = nullptr;
     void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled entry point
+    // tensor maps of the last encode call (6 x 128 bytes, 64-byte aligned) and what they describe
+    alignas(64) unsigned char tmaps[AGC_ENC_BOX_SIZES * 128];
+    const float *tmaps_G = nullptr;
+    long long tmaps_ld = 0;
 };
 
 int agc_launch_encode(agc_plan *plan, const float *G, const float *const *G_rows, long long ld, uint64_t round,
