@@ -10,6 +10,10 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+    # the shared library is a build product (not in the history): compile it when it is missing or
+    # older than its sources, so that a fresh checkout can run the suite directly
+    from paper_2605_15890_b200 import build as lib_build
+    lib_build.build()
 
 
 def _have_gpu():
