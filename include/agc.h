@@ -144,8 +144,8 @@ int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64
  * agc_encode_quantize_rows - the same round for partial gradients that live in k separate
  * device buffers (one per partition, e.g. the flat gradients of k model replicas).
  *
- *   G_rows_dev device, k pointers to device rows of at least d fp32 each; every row 16-byte
- *              aligned (checked by the kernel's loads: a misaligned row is a caller error)
+ *   G_rows_dev device, k pointers to device rows of at least d fp32 each; rows that are
+ *              16-byte aligned are read with 128-bit loads, others element by element
  * Everything else as agc_encode_quantize; same messages, bit for bit. Without a common base
  * and stride the rows cannot be described by one tensor map, so this call uses the direct-load
  * kernel: the replicas of a partition are re-read through L2 instead of being staged once.

@@ -657,7 +657,11 @@ def test_encode_from_separate_row_buffers(agc, torch, B):
     G = torch.from_numpy(G_host).cuda()
     ses.encode(G, 6)
     want_codes, want_scales = ses.codes.clone(), ses.scales.clone()
-    rows = [torch.from_numpy(G_host[j].copy()).cuda() for j in reversed(range(k))][::-1]   # separate allocations
+    # separate allocations; every other row starts 4 bytes into its buffer (not 16-byte aligned)
+    bufs = [torch.zeros(d + 4, dtype=torch.float32, device="cuda") for _ in range(k)]
+    rows = [bufs[j][(j & 1):(j & 1) + d] for j in range(k)]
+    for j in range(k):
+        rows[j].copy_(torch.from_numpy(G_host[j]))
     ptrs = torch.tensor([r.data_ptr() for r in rows], dtype=torch.int64, device="cuda")
     ses.codes.fill_(-1)
     ses.scales.fill_(-1.0)
