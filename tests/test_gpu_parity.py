@@ -497,19 +497,27 @@ def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
     ses.close()
 
 
-def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch):
+@pytest.mark.parametrize("kind", ["cyclic", "interval"])
+def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch, kind):
     """Lemma 1 as a measured experiment: 20 rounds x 64 straggler realisations through the CUDA
     path (fresh rounding each round, fresh Bernoulli masks each realisation). The mean of
     g_hat approaches sum_j g_j (unbiasedness, Eq. exp_g2_quant) and the mean squared error
-    stays below C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 with ||g_j||^2 = C."""
+    stays below C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 with ||g_j||^2 = C. With
+    the paper's interval construction (the optimal structure of Theorem 1) that bound is
+    Lemma 2's k^2 C / sum_i c_i^-1."""
     from paper_2605_15890_b200.session import Session
     rng = np.random.default_rng(31)
     n = k = 8
     d, B = 4096, 512
     bits = np.array([2, 3, 4, 6, 2, 5, 3, 4], np.uint8)
     p = rng.uniform(0.05, 0.4, n)
-    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B)
+    if kind == "cyclic":
+        rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, B)
+    else:
+        rp, ci, a, w = _codes.interval_code(p, bits, k, B)
     A = od.csr_to_dense(rp, ci, a.astype(np.float64), k)
+    if kind == "interval":
+        assert np.isclose(od.lemma1_bound(A, w.astype(np.float64), p, bits, B), od.lemma2_bound(p, bits, k, B), rtol=1e-5)
     G_host = rng.standard_normal((k, d)).astype(np.float32)
     G_host /= np.linalg.norm(G_host.astype(np.float64), axis=1, keepdims=True).astype(np.float32)   # C = 1
     g = G_host.astype(np.float64).sum(axis=0)
