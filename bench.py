@@ -140,6 +140,39 @@ def oracle_round(orp, code, bits, bucket, seed, t, G, d, mask, lr, beta):
     return beta
 
 
+def parity_sample(ses, G, wl, code, bits, bucket, blocks=(0, 1, 2, 3)):
+    """The messages the GPU produced for the bench's own inputs against the oracle on a few pack
+    blocks (first ones and the last): counts of differing code words and scales (expected 0).
+    Bucket-wise mode only (the global norm needs the whole vector)."""
+    if not bucket:
+        return None
+    from oracle import roundpath as orp
+    rp, ci, a, w = code
+    nblk = (wl.d + 511) // 512
+    rnd = 12345
+    ses.encode(G, rnd)
+    off = orp.worker_word_offsets(wl.d, bits)
+    bad_codes = bad_scales = 0
+    qs = sorted({q for q in blocks if q < nblk} | {nblk - 1})
+    for q in qs:
+        m0, m1 = q * 512, min((q + 1) * 512, wl.d)
+        blk = np.zeros((wl.k, 512), np.float32)
+        blk[:, :m1 - m0] = G[:, m0:m1].cpu().numpy()
+        oc, osc, _, _ = orp.encode_block(rp, ci, a, bits, bucket, wl.seed, rnd, q + ses.first_block, blk)
+        wb = 0
+        for i in range(wl.n):
+            b = int(bits[i])
+            lo = int(off[i]) + q * 16 * b
+            got = ses.codes[lo:lo + 16 * b].cpu().numpy().view(np.uint32)
+            bad_codes += int((got != oc[wb:wb + 16 * b]).sum())
+            wb += 16 * b
+        per = 512 // bucket
+        nb = (wl.d + bucket - 1) // bucket
+        got_s = ses.scales.view(wl.n, -1)[:, q * per:min((q + 1) * per, nb)].cpu().numpy()
+        bad_scales += int((got_s.view(np.uint32) != osc[:, :got_s.shape[1]].view(np.uint32)).sum())
+    return {"pack_blocks": qs, "code_words_differ": bad_codes, "scales_differ": bad_scales}
+
+
 def oracle_sample_rate(wl, code, bits, bucket, target_s=12.0):
     """Time the CPU oracle (as it stands, one thread) on a bounded sample of the workload:
     whole pack blocks through encode + quantise + pack + decode + update."""
@@ -390,6 +423,7 @@ def main():
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                                     "sample": f"{d_s} of {wl.d} coordinates (whole pack blocks, all {wl.n} workers), "
                                               f"one round, {secs:.1f} s"}
+            line["parity_sample"] = parity_sample(ses, G, wl, code, bits, bucket)
         print(json.dumps(line))
     ses.close()
     if dist:

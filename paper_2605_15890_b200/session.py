@@ -22,10 +22,12 @@ class Session:
                                   device=self.device)
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.uses_tma = B.agc_plan_uses_tma(self.plan)
+        self.first_block = 0
 
     def set_first_block(self, first_block):
         """Place this plan's coordinates at pack block `first_block` of a longer vector."""
         B.agc_plan_set_first_block(self.plan, first_block)
+        self.first_block = first_block
 
     def close(self):
         if self.plan is not None:
