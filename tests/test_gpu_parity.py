@@ -106,9 +106,9 @@ def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
     assert out["tma"] == (not direct)
 
 
-@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered"])
+@pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered", "thousands"])
 def test_code_structures(agc, torch, kind):
-    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered"].index(kind))
+    rng = np.random.default_rng(["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered", "thousands"].index(kind))
     d = 3000
     if kind == "identity":
         n = k = 5
@@ -135,6 +135,12 @@ def test_code_structures(agc, torch, kind):
         bits = rng.integers(2, 9, n).astype(np.uint8)
         p = rng.uniform(0.05, 0.5, n)
         code = _codes.cyclic_code(p, bits, k, 40, 512)
+    elif kind == "thousands":      # more workers than the staged kernels' tables hold: both fall back
+        n = k = 2100
+        d = 700
+        bits = rng.integers(1, 9, n).astype(np.uint8)
+        p = rng.uniform(0.01, 0.5, n)
+        code = _codes.cyclic_code(p, bits, k, 2, 512)
     elif kind == "scattered":      # supports scattered over the partitions (not banded): clustered groups
         n, k = 60, 90
         bits = rng.integers(1, 9, n).astype(np.uint8)
@@ -161,7 +167,7 @@ def test_code_structures(agc, torch, kind):
     masks = (rng.random((1, n)) >= p).astype(np.uint8)
     out, ref = run_both(agc, torch, G, code, p, bits, 512, 77, 3, masks)
     assert_exact(out, ref)
-    assert out["tma"] == (kind != "wide_rows")
+    assert out["tma"] == (kind not in ("wide_rows", "thousands"))
     assert G.shape[0] == k
 
 
