@@ -500,6 +500,16 @@ def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
     og, ob = orp.decode(d, bits, 512, w, mask[None], oc, orp.expand_global_scales(osc, d), lr=lr, beta=beta0)
     assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
     assert (beta.cpu().numpy().view(np.uint32) == ob.view(np.uint32)).all()
+    if not direct:
+        # the two-track decoder reads the same single scale per worker
+        v2 = (0.5 * w).astype(np.float32)
+        gw = torch.empty(d, dtype=torch.float32, device="cuda")
+        gv = torch.empty(d, dtype=torch.float32, device="cuda")
+        agc.agc_decode_two_track(ses.plan, ses.codes, ses.scales, torch.from_numpy(mask).cuda(), v2, gw, gv,
+                                 status_dev=ses.status)
+        ogv, _ = orp.decode(d, bits, 512, v2, mask[None], oc, orp.expand_global_scales(osc, d))
+        assert (gw.cpu().numpy().view(np.uint32) == og[0].view(np.uint32)).all()
+        assert (gv.cpu().numpy().view(np.uint32) == ogv[0].view(np.uint32)).all()
     ses.close()
 
 
