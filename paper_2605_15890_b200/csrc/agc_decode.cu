@@ -292,22 +292,40 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
             for (int t = 0; t <= H; ++t) A[t] = W[t];
         }
     }
+    // two coordinates at a time: the subtraction and the fma are packed instructions (two
+    // independent IEEE fp32 operations each), which halves their issue slots
 #pragma unroll
-    for (int t = 0; t < 16; ++t) {
-        const int bitpos = t * BITS;
-        const int w = bitpos >> 5, sh = bitpos & 31;
-        float level;
-        if constexpr (BITS == 1) {
-            level = __uint_as_float(0xBF000000u ^ ((A[0] >> t) << 31));                     // code - 0.5
-        } else {
-            uint32_t x;
-            if constexpr (BITS == 8) x = __byte_perm(A[w], 0x4B000000u, 0x7540u | (uint32_t)(sh >> 3));
-            else if (sh + BITS <= 32) x = and_or(sh ? A[w] >> sh : A[w], MASK, 0x4B000000u);
-            else x = and_or(__funnelshift_r(A[w], A[w + 1], sh), MASK, 0x4B000000u);
-            level = __fsub_rn(__uint_as_float(x), 8388608.0f + (float)L);                   // code - L, exact
+    for (int t = 0; t < 16; t += 2) {
+        float lv[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int bitpos = (t + h) * BITS;
+            const int w = bitpos >> 5, sh = bitpos & 31;
+            if constexpr (BITS == 1) {
+                lv[h] = __uint_as_float(0xBF000000u ^ ((A[0] >> (t + h)) << 31));              // code - 0.5
+            } else {
+                uint32_t x;
+                if constexpr (BITS == 8) x = __byte_perm(A[w], 0x4B000000u, 0x7540u | (uint32_t)(sh >> 3));
+                else if (sh + BITS <= 32) x = and_or(sh ? A[w] >> sh : A[w], MASK, 0x4B000000u);
+                else x = and_or(__funnelshift_r(A[w], A[w + 1], sh), MASK, 0x4B000000u);
+                lv[h] = __uint_as_float(x);                                                    // 2^23 + code
+            }
         }
-        acc[t] = __fmaf_rn(cstep_row[t >> 2], level, acc[t]);
-        if constexpr (TWO) acc2[t] = __fmaf_rn(cstep2_row[t >> 2], level, acc2[t]);
+        float2 level = make_float2(lv[0], lv[1]);
+        if constexpr (BITS >= 2) {
+            constexpr float NEG = -(8388608.0f + (float)L);
+            level = __fadd2_rn(level, make_float2(NEG, NEG));                                  // code - L, exact
+        }
+        const float c = cstep_row[t >> 2];
+        const float2 r = __ffma2_rn(make_float2(c, c), level, make_float2(acc[t], acc[t + 1]));
+        acc[t] = r.x;
+        acc[t + 1] = r.y;
+        if constexpr (TWO) {
+            const float c2 = cstep2_row[t >> 2];
+            const float2 r2 = __ffma2_rn(make_float2(c2, c2), level, make_float2(acc2[t], acc2[t + 1]));
+            acc2[t] = r2.x;
+            acc2[t + 1] = r2.y;
+        }
     }
 }
 
