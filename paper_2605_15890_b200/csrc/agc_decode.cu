@@ -391,6 +391,11 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     extern __shared__ __align__(1024) unsigned char smem[];
     const int stages = P.stages;
     const uint32_t stage_bytes = QT * 64u * AGC_DEC_GROUP_BITS;
+    // Tile height of this launch: QT blocks for long vectors, fewer when the vector has too
+    // few blocks to give every SM a full tile. A shorter tile leaves room in a stage for a
+    // wider group of workers, so that a short vector passes the ring in fewer steps.
+    const uint32_t qt = (uint32_t)P.qt;
+    const uint32_t cap_bits = AGC_DEC_GROUP_BITS * QT / qt;
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)stages * stage_bytes);
     uint64_t *empty = full + AGC_DEC_MAX_STAGES;
     volatile int *flags = reinterpret_cast<volatile int *>(empty + AGC_DEC_MAX_STAGES);  // abort x2, n_groups
@@ -433,7 +438,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     __syncthreads();
     if (threadIdx.x == 0) {
         // compact list of the workers that contribute, cut into groups of at most 32 workers
-        // and AGC_DEC_GROUP_BITS bits per coordinate
+        // and as many bits per coordinate as a stage holds for a tile of qt blocks
         int nrecv = 0, ng = 0, in_grp = 0, run_head = 0;
         uint32_t grp_bits = 0, soff = 0;
         long long word_off = 0;
@@ -443,7 +448,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
             const long long my_off = word_off;
             word_off += P.nblk * 16 * (long long)s_raw_allb[i];
             if (b == 0) continue;
-            if (in_grp == 32 || grp_bits + b > AGC_DEC_GROUP_BITS) {
+            if (in_grp == 32 || grp_bits + b > cap_bits) {
                 s_grp_ptr[++ng] = nrecv;
                 in_grp = 0; grp_bits = 0; soff = 0;
             }
@@ -461,7 +466,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
             wk.run = 1;
             if (TWO) s_w2[nrecv] = P.v[i];
             s_wk[nrecv++] = wk;
-            soff += QT * 64u * b;
+            soff += qt * 64u * b;
             grp_bits += b;
             ++in_grp;
         }
@@ -470,7 +475,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     }
     __syncthreads();
     const int n_groups = flags[2];
-    const long long ntile = (P.nblk + QT - 1) / QT;
+    const long long ntile = (P.nblk + qt - 1) / qt;
 
     if (warp == QT) {
         // ---------------- producer
@@ -479,8 +484,8 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         uint32_t parity = 1;
         bool ok = true;
         for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q0 = T * QT;
-            const uint32_t nq = (uint32_t)(P.nblk - q0 < QT ? P.nblk - q0 : QT);
+            const long long q0 = T * qt;
+            const uint32_t nq = (uint32_t)(P.nblk - q0 < qt ? P.nblk - q0 : qt);
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 uint32_t bytes = 0, soff = 0, wbits = 0;
@@ -504,10 +509,10 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
 #if AGC_DEC_PREFETCH
                     // the same workers' chunks of this CTA's next tile row: on their way to L2 a
                     // whole tile row ahead, so that the ring refills at L2 latency, not HBM latency
-                    const long long qn = q0 + (long long)gridDim.x * QT;
+                    const long long qn = q0 + (long long)gridDim.x * qt;
                     if (qn < P.nblk) {
-                        const uint32_t nqn = (uint32_t)(P.nblk - qn < QT ? P.nblk - qn : QT);
-                        bulk_prefetch_l2(src + (size_t)gridDim.x * QT * 64u * wbits, nqn * 64u * wbits);
+                        const uint32_t nqn = (uint32_t)(P.nblk - qn < qt ? P.nblk - qn : qt);
+                        bulk_prefetch_l2(src + (size_t)gridDim.x * qt * 64u * wbits, nqn * 64u * wbits);
                     }
 #endif
                 }
@@ -532,8 +537,8 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         auto fetch_scales = [&](long long T, int g, float (&sc)[4 / RB]) {
 #pragma unroll
             for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
-            const long long q = T * QT + warp;
-            if (T < ntile && g < n_groups && q < P.nblk) {
+            const long long q = T * qt + warp;
+            if (T < ntile && g < n_groups && (uint32_t)warp < qt && q < P.nblk) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 if (lane < nr) {
                     const float *srow = P.scales + s_wk[r0 + lane].scales_off;
@@ -548,8 +553,8 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         float sc_next[4 / RB];
         fetch_scales(blockIdx.x, 0, sc_next);
         for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q = T * QT + warp;
-            const bool active = q < P.nblk;
+            const long long q = T * qt + warp;
+            const bool active = (uint32_t)warp < qt && q < P.nblk;
             float acc[16], acc2[16], b[16];   // acc2: second track, unused and dropped in the other modes
 #pragma unroll
             for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
@@ -669,6 +674,14 @@ bool ring_set_smem(int smem)
            cudaFuncSetAttribute(agc_decode_ring_kernel<1, MODE, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) == cudaSuccess;
 }
 
+// Blocks per tile of a ring launch: the full height when every SM gets at least one full
+// tile, else the vector's blocks spread evenly over the SMs.
+int ring_tile_height(long long nblk, int sm_count, int qt_max)
+{
+    const long long even = (nblk + sm_count - 1) / sm_count;
+    return (int)(even < 1 ? 1 : (even < qt_max ? even : qt_max));
+}
+
 template <bool COLLAPSED>
 void launch(const AgcDecParams &P, int grid, cudaStream_t stream)
 {
@@ -716,7 +729,8 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
         P.weff = plan->d_weff;
     }
     if (plan->dec_ring) {
-        const long long ntile = (plan->nblk + AGC_DEC_QT - 1) / AGC_DEC_QT;
+        P.qt = ring_tile_height(plan->nblk, plan->sm_count, AGC_DEC_QT);
+        const long long ntile = (plan->nblk + P.qt - 1) / P.qt;
         const int grid = (int)(ntile < plan->sm_count ? ntile : plan->sm_count);
         if (collapsed) {
             if (launch_ring<1, AGC_DEC_QT>(P, grid, plan->dec_smem, stream) != cudaSuccess) return AGC_ERR_CUDA;
@@ -797,7 +811,8 @@ int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *
         P.adam_ibc1 = float(1.0 / (1.0 - std::pow(b1, double(adam->step))));
         P.adam_ibc2 = float(1.0 / (1.0 - std::pow(b2, double(adam->step))));
     }
-    const long long ntile = (plan->nblk + AGC_DEC_QT2 - 1) / AGC_DEC_QT2;
+    P.qt = ring_tile_height(plan->nblk, plan->sm_count, AGC_DEC_QT2);
+    const long long ntile = (plan->nblk + P.qt - 1) / P.qt;
     const int grid = (int)(ntile < plan->sm_count ? ntile : plan->sm_count);
     return launch_ring<2, AGC_DEC_QT2>(P, grid, plan->dec2_smem, stream) == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
 }

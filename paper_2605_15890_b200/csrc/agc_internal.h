@@ -103,6 +103,7 @@ struct AgcDecParams {
     const float *lr;        // device, R learning rates (per-realisation mode with beta)
     uint32_t *status = nullptr;  // AGC_STATUS_* bits are OR-ed into it (ring kernel), may be NULL
     int stages = 0;              // ring depth of the ring kernel
+    int qt = 1;                  // blocks per tile of this ring launch (at most the kernel's QT)
     uint32_t w2_offset = 0;      // byte offset of the second-decoder array in shared memory
     // two-track decode
     const float *v = nullptr;    // n second decoding coefficients
