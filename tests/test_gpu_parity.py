@@ -171,6 +171,46 @@ def test_code_structures(agc, torch, kind):
     assert G.shape[0] == k
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_seeded_random_shapes_codes_and_masks(agc, torch, case):
+    """Random worker / partition counts, sparse supports, widths, bucket sizes, lengths (a few
+    blocks up to several hundred: every tile height of the decoder), heavy-tailed values, 64-bit
+    seeds and round numbers, several realisations with the fused update."""
+    rng = np.random.default_rng(9000 + case)
+    n = int(rng.integers(1, 70))
+    k = int(rng.integers(1, 50))
+    B = int(rng.choice([128, 256, 512]))
+    d = int(rng.choice([rng.integers(1, 3000), rng.integers(3000, 80_000), rng.integers(80_000, 400_000)]))
+    if n * d > 6_000_000:
+        d = 6_000_000 // n
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.0, 0.7, n)
+    rp = [0]
+    ci, a = [], []
+    for i in range(n):
+        cols = np.sort(rng.choice(k, size=int(rng.integers(1, min(k, 6) + 1)), replace=False))
+        ci.extend(cols.tolist())
+        a.extend((rng.standard_normal(cols.size) * 10.0 ** rng.uniform(-2, 1)).tolist())
+        rp.append(len(ci))
+    code = (np.array(rp, np.int32), np.array(ci, np.int32), np.array(a, np.float32),
+            (rng.standard_normal(n) * 2).astype(np.float32))
+    G = (rng.standard_t(3, (k, d)) * 10.0 ** rng.uniform(-4, 3, (k, 1))).astype(np.float32)
+    if case % 4 == 0:
+        G[rng.integers(0, k), : min(d, 600)] = 0.0          # stretches of zeros inside a row
+    R = int(rng.integers(1, 5))
+    masks = (rng.random((R, n)) >= p).astype(np.uint8)
+    lr = rng.uniform(1e-3, 1e-1, R).astype(np.float32)
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    seed = int(rng.integers(0, 2**63)) * 2 + 1
+    rnd = int(rng.integers(0, 2**63))
+    out, ref = run_both(agc, torch, G, code, p, bits, B, seed, rnd, masks, lr=lr, beta0=beta0,
+                        ld_pad=int(rng.choice([0, 4, 36])))
+    assert_exact(out, ref)
+    assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
+    scale = max(np.abs(ref["beta"]).max(), 1e-30)
+    assert np.abs(out["beta_fused"] - ref["beta"]).max() / scale <= 1e-5
+
+
 def test_straggler_extremes_and_batched_decode(agc, torch):
     """All stragglers (g_hat = 0), none, single survivors; R realisations with per-
     realisation outputs, the sequential update and the collapsed update."""
