@@ -637,6 +637,233 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     if (threadIdx.x == 0 && (flags[0] || flags[1]) && P.status) atomicOr(P.status, AGC_STATUS_TIMEOUT);
 }
 
+// ------------------------------------------------------------------ many realisations, g_hat of each
+// g_hat^(r) = sum_i I_{r,i} w_i v_i for a chunk of up to 64 realisations in one pass over the
+// messages: every received worker's block is unpacked once (levels as floats in shared
+// memory), then each thread adds it to its 16 realisations x 4 coordinates with the
+// coefficient c_{r,i} = I_{r,i} * (w_i S_i / L_i) of each realisation. A coefficient of zero
+// leaves the sum as it is, so every realisation sees exactly the fmas of its own workers, in
+// ascending worker order: the result equals the realisation-by-realisation decode bit for bit.
+// CTA = 4 rows of 128 coordinates x RG groups of 16 realisations, one warp each; the warps
+// take turns by batches of W = 4 RG workers: each unpacks one worker of the batch, then
+// all add the whole batch.
+struct __align__(16) AgcMultiWorker {
+    long long word_off;      // word offset of the worker's message
+    unsigned long long rmask;  // bit r: realisation r of the chunk received this worker
+    float weight;            // w_i
+    int worker;
+    int bits;
+    int pad;
+};
+
+// The lane's 16 levels (code - L, or code - 1/2 for one-bit codes) from its words of the block.
+template <int BITS>
+__device__ __forceinline__ void multi_levels(const uint32_t (&W)[4], int lane, float (&lv)[16])
+{
+    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+    constexpr int NACC = (16 * BITS + 31) / 32;
+    uint32_t A[NACC + 1];
+    A[NACC] = 0u;
+    if constexpr (BITS % 2 == 0) {
+#pragma unroll
+        for (int t = 0; t < NACC; ++t) A[t] = W[t];
+    } else {
+        constexpr int H = (BITS - 1) / 2;
+        if (lane & 1) {
+#pragma unroll
+            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
+            A[H] = W[H] >> 16;
+        } else {
+#pragma unroll
+            for (int t = 0; t <= H; ++t) A[t] = W[t];
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+        const int bitpos = t * BITS;
+        const int w = bitpos >> 5, sh = bitpos & 31;
+        uint32_t code;
+        if (sh + BITS <= 32) code = (A[w] >> sh) & MASK;
+        else code = __funnelshift_r(A[w], A[w + 1], sh) & MASK;
+        if constexpr (BITS >= 2)
+            lv[t] = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);  // code - L, exact
+        else
+            lv[t] = __uint_as_float(0xBF000000u ^ (code << 31));                          // code - 0.5
+    }
+}
+
+template <int RB>
+__global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecParams P, int r0, int Rc)
+{
+    extern __shared__ __align__(16) unsigned char multi_smem[];
+    const int W = blockDim.x >> 5;   // warps = workers per batch
+    float *s_levels = reinterpret_cast<float *>(multi_smem);                            // [2][W][512]
+    float *s_coef = s_levels + 2 * W * AGC_BLOCK;                                       // [2][W][4 / RB][64]
+    AgcMultiWorker *s_list = reinterpret_cast<AgcMultiWorker *>(s_coef + 2 * W * (4 / RB) * 64);
+    unsigned long long *s_rmask = reinterpret_cast<unsigned long long *>(s_list + P.n);  // per worker, before compaction
+    int *s_nrecv = reinterpret_cast<int *>(s_rmask + P.n);
+
+    const int wp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = wp & 3, rg = wp >> 2;
+    // which realisations of the chunk received each worker
+    for (int i = threadIdx.x; i < P.n; i += blockDim.x) {
+        unsigned long long m = 0ull;
+        for (int r = 0; r < Rc; ++r)
+            if (P.masks[(long long)(r0 + r) * P.n + i]) m |= 1ull << r;
+        s_rmask[i] = m;
+    }
+    __syncthreads();
+    if (wp == 0) {
+        // ascending list of the workers that some realisation received
+        int cnt = 0;
+        for (int base = 0; base < P.n; base += 32) {
+            const int i = base + lane;
+            const unsigned long long m = i < P.n ? s_rmask[i] : 0ull;
+            const unsigned vote = __ballot_sync(0xffffffffu, m != 0ull);
+            if (m != 0ull) {
+                AgcMultiWorker e;
+                e.word_off = P.word_off[i];
+                e.rmask = m;
+                e.weight = P.w[i];
+                e.worker = i;
+                e.bits = P.bits[i];
+                e.pad = 0;
+                s_list[cnt + __popc(vote & ((1u << lane) - 1u))] = e;
+            }
+            cnt += __popc(vote);
+        }
+        if (lane == 0) *s_nrecv = cnt;
+    }
+    __syncthreads();
+    const int nrecv = *s_nrecv;
+    const int nbatch = (nrecv + W - 1) / W;
+    const bool vec = (P.d & 3) == 0;
+
+    // words and scales of the worker this warp unpacks next, fetched one batch ahead
+    uint32_t pw[4];
+    float ps[4 / RB];
+    int pidx = -1;
+    auto prefetch = [&](long long q, int b) {
+        pidx = -1;
+        if (q >= P.nblk || b >= nbatch) return;
+        const int idx = b * W + wp;
+        if (idx >= nrecv) return;
+        pidx = idx;
+        const AgcMultiWorker e = s_list[idx];
+        const uint32_t *blk = P.codes + e.word_off + q * 16 * e.bits;
+        const uint32_t *src;
+        int cnt;
+        if (e.bits & 1) {
+            const int H = (e.bits - 1) >> 1;
+            src = blk + (lane >> 1) * e.bits + ((lane & 1) ? H : 0);
+            cnt = H + 1;
+        } else {
+            cnt = e.bits >> 1;
+            src = blk + lane * cnt;
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) pw[t] = t < cnt ? __ldg(src + t) : 0u;
+#pragma unroll
+        for (int bk = 0; bk < 4 / RB; ++bk) {
+            const long long beta_idx = P.global_norm ? 0 : q * (4 / RB) + bk;
+            ps[bk] = beta_idx < P.nb ? __ldg(P.scales + (long long)e.worker * P.nb + beta_idx) : 0.0f;
+        }
+    };
+
+    prefetch(blockIdx.x, 0);
+    int it = 0;   // batches so far: consecutive batches alternate between the two buffers, across blocks too
+    for (long long q = blockIdx.x; q < P.nblk; q += gridDim.x) {
+        float2 acc[8][4];   // [pair of realisations][coordinate]
+#pragma unroll
+        for (int pr = 0; pr < 8; ++pr)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[pr][e] = make_float2(0.0f, 0.0f);
+        for (int b = 0; b < nbatch; ++b, ++it) {
+            const int buf = it & 1;
+            if (pidx >= 0) {
+                // unpack this warp's worker of the batch and form its coefficients
+                const AgcMultiWorker e = s_list[pidx];
+                float lv[16];
+                switch (e.bits) {
+                    case 1: multi_levels<1>(pw, lane, lv); break;
+                    case 2: multi_levels<2>(pw, lane, lv); break;
+                    case 3: multi_levels<3>(pw, lane, lv); break;
+                    case 4: multi_levels<4>(pw, lane, lv); break;
+                    case 5: multi_levels<5>(pw, lane, lv); break;
+                    case 6: multi_levels<6>(pw, lane, lv); break;
+                    case 7: multi_levels<7>(pw, lane, lv); break;
+                    default: multi_levels<8>(pw, lane, lv); break;
+                }
+                float *dst = s_levels + ((size_t)buf * W + wp) * AGC_BLOCK + 4 * lane;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<float4 *>(dst + 128 * c) = make_float4(lv[4 * c], lv[4 * c + 1], lv[4 * c + 2], lv[4 * c + 3]);
+                const float dstep = e.bits >= 2 ? (float)(1.0 / (double)((1 << (e.bits - 1)) - 1)) : 2.0f;
+                float *cdst = s_coef + ((size_t)buf * W + wp) * (4 / RB) * 64;
+#pragma unroll
+                for (int bk = 0; bk < 4 / RB; ++bk) {
+                    const float cs = __fmul_rn(__fmul_rn(e.weight, ps[bk]), dstep);
+                    cdst[bk * 64 + lane] = ((e.rmask >> lane) & 1ull) ? cs : 0.0f;
+                    cdst[bk * 64 + 32 + lane] = ((e.rmask >> (32 + lane)) & 1ull) ? cs : 0.0f;
+                }
+            }
+            if (b + 1 < nbatch) prefetch(q, b + 1);
+            else prefetch(q + gridDim.x, 0);
+            // one barrier per batch: a buffer is rewritten two batches later, after the barrier
+            // of the batch in between, which no warp passes before it has finished this one
+            __syncthreads();
+            const int cntb = nrecv - b * W < W ? nrecv - b * W : W;
+            const float *lsrc = s_levels + (size_t)buf * W * AGC_BLOCK + 128 * row + 4 * lane;
+            const float *csrc = s_coef + (size_t)buf * W * (4 / RB) * 64 + (row / RB) * 64 + 16 * rg;
+            for (int j = 0; j < cntb; ++j) {
+                const float4 l4 = *reinterpret_cast<const float4 *>(lsrc + (size_t)j * AGC_BLOCK);
+                const float4 *cp = reinterpret_cast<const float4 *>(csrc + (size_t)j * (4 / RB) * 64);
+                const float4 c0 = cp[0], c1 = cp[1], c2 = cp[2], c3 = cp[3];
+                const float2 cpair[8] = {make_float2(c0.x, c0.y), make_float2(c0.z, c0.w), make_float2(c1.x, c1.y),
+                                         make_float2(c1.z, c1.w), make_float2(c2.x, c2.y), make_float2(c2.z, c2.w),
+                                         make_float2(c3.x, c3.y), make_float2(c3.z, c3.w)};
+                const float lvs[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 l2 = make_float2(lvs[e], lvs[e]);
+#pragma unroll
+                    for (int pr = 0; pr < 8; ++pr) acc[pr][e] = __ffma2_rn(cpair[pr], l2, acc[pr][e]);
+                }
+            }
+        }
+        // realisations 16 rg .. 16 rg + 15 of the chunk, coordinates 128 row + 4 lane .. + 3 of block q
+        const long long m0 = q * AGC_BLOCK + 128 * row + 4 * lane;
+#pragma unroll
+        for (int pr = 0; pr < 8; ++pr) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int r = 16 * rg + 2 * pr + h;
+                if (r >= Rc) continue;
+                float *out = P.ghat + (long long)(r0 + r) * P.d + m0;
+                const float v0 = h ? acc[pr][0].y : acc[pr][0].x, v1 = h ? acc[pr][1].y : acc[pr][1].x;
+                const float v2 = h ? acc[pr][2].y : acc[pr][2].x, v3 = h ? acc[pr][3].y : acc[pr][3].x;
+                if (vec && m0 + 3 < P.d) {
+                    *reinterpret_cast<float4 *>(out) = make_float4(v0, v1, v2, v3);
+                } else {
+                    if (m0 < P.d) out[0] = v0;
+                    if (m0 + 1 < P.d) out[1] = v1;
+                    if (m0 + 2 < P.d) out[2] = v2;
+                    if (m0 + 3 < P.d) out[3] = v3;
+                }
+            }
+        }
+    }
+}
+
+// Shared memory of the kernel above for RG groups of 16 realisations and n workers.
+size_t multi_smem_bytes(int rg, int rows_per_bucket, int n)
+{
+    const size_t W = 4 * size_t(rg);
+    return sizeof(float) * 2 * W * AGC_BLOCK + sizeof(float) * 2 * W * (4 / rows_per_bucket) * 64 +
+           sizeof(AgcMultiWorker) * size_t(n) + sizeof(unsigned long long) * size_t(n) + 16;
+}
+
 template <int MODE, int QT>
 cudaError_t launch_ring(const AgcDecParams &P, int grid, size_t smem, cudaStream_t stream)
 {
@@ -680,6 +907,28 @@ int ring_tile_height(long long nblk, int sm_count, int qt_max)
 {
     const long long even = (nblk + sm_count - 1) / sm_count;
     return (int)(even < 1 ? 1 : (even < qt_max ? even : qt_max));
+}
+
+// g_hat of R >= AGC_DEC_MULTI_MIN_R realisations: chunks of up to 64 realisations per launch.
+template <int RB>
+int launch_multi_rb(const AgcDecParams &P, int sm_count, int smem_optin, cudaStream_t stream)
+{
+    for (int r0 = 0; r0 < P.R; r0 += 64) {
+        const int Rc = P.R - r0 < 64 ? P.R - r0 : 64;
+        const int rg = (Rc + 15) / 16;
+        const int threads = 128 * rg;
+        const size_t smem = multi_smem_bytes(rg, RB, P.n);
+        if (smem > size_t(smem_optin)) return AGC_ERR_STATE;
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agc_decode_multi_kernel<RB>, threads, smem) != cudaSuccess ||
+            per_sm < 1)
+            return AGC_ERR_CUDA;
+        const long long slots = (long long)sm_count * per_sm;
+        const int grid = (int)(P.nblk < slots ? P.nblk : slots);
+        agc_decode_multi_kernel<RB><<<grid, threads, smem, stream>>>(P, r0, Rc);
+        if (cudaGetLastError() != cudaSuccess) return AGC_ERR_CUDA;
+    }
+    return AGC_OK;
 }
 
 template <bool COLLAPSED>
@@ -728,6 +977,12 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
                                                                                plan->d_weff);
         P.weff = plan->d_weff;
     }
+    if (plan->dec_ring && ghat && !beta && R >= AGC_DEC_MULTI_MIN_R &&
+        multi_smem_bytes(4, P.rows_per_bucket, plan->n) <= size_t(plan->smem_optin)) {
+        if (P.rows_per_bucket == 4) return launch_multi_rb<4>(P, plan->sm_count, plan->smem_optin, stream);
+        if (P.rows_per_bucket == 2) return launch_multi_rb<2>(P, plan->sm_count, plan->smem_optin, stream);
+        return launch_multi_rb<1>(P, plan->sm_count, plan->smem_optin, stream);
+    }
     if (plan->dec_ring) {
         P.qt = ring_tile_height(plan->nblk, plan->sm_count, AGC_DEC_QT);
         const long long ntile = (plan->nblk + P.qt - 1) / P.qt;
@@ -762,6 +1017,11 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
     if (!ring_set_smem<0, AGC_DEC_QT>(int(plan->dec_smem)) || !ring_set_smem<1, AGC_DEC_QT>(int(plan->dec_smem)) ||
         !ring_set_smem<2, AGC_DEC_QT2>(int(plan->dec2_smem)))
         return AGC_ERR_CUDA;
+    if (cudaFuncSetAttribute(agc_decode_multi_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    plan->smem_optin = smem_optin;
     plan->dec_ring = true;
     return AGC_OK;
 }

@@ -27,6 +27,7 @@
 #endif
 #define AGC_DEC_MAX_STAGES 8
 #define AGC_DEC_QT2 23         // consumer warps of the two-track decoder (two accumulator sets: 80 registers)
+#define AGC_DEC_MULTI_MIN_R 8    // from this many realisations on, g_hat of all of them comes from one pass over the messages
 #define AGC_DEC_RING_MAX_WORKERS 2048  // above this the per-worker tables no longer fit shared memory
 #define AGC_STATIC_MAX_WORKERS 1024  // limits of the allocation-free update
 #define AGC_STATIC_MAX_R 4096
@@ -132,6 +133,7 @@ struct agc_plan {
     size_t enc_smem = 0;
     // decode ring
     bool dec_ring = false;
+    int smem_optin = 0;           // largest dynamic shared memory of a CTA on the plan's device
     int dec_stages = 0;
     size_t dec_smem = 0;
     int dec2_stages = 0;

@@ -553,6 +553,43 @@ def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
     ses.close()
 
 
+@pytest.mark.parametrize("R,B,d,n", [(8, 512, 5000, 12), (16, 256, 70_001, 9), (17, 128, 1300, 40), (33, 512, 513, 70),
+                                     (64, 512, 200_000, 20), (65, 256, 4097, 33), (130, 128, 3, 5), (48, 0, 40_000, 6)])
+def test_g_hat_of_many_realisations_in_one_pass(agc, torch, R, B, d, n):
+    """From 8 realisations on, g_hat of every realisation comes from one pass over the messages
+    (chunks of 64 realisations). Every row must equal the oracle's realisation-by-realisation
+    decode bit for bit; rows with no survivor and workers nobody received are in the masks."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(R * 1000 + n)
+    k = n
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.6, n)
+    masks = (rng.random((R, n)) >= p).astype(np.uint8)
+    masks[R // 2] = 0                       # a realisation in which every worker straggles
+    masks[:, n // 3] = 0                    # a worker that no realisation receives
+    masks[R - 1] = 1
+    masks[R - 1, n // 3] = 0
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-3, 2, (k, 1))).astype(np.float32)
+    if B:
+        code = _codes.cyclic_code(p, bits, k, min(3, k), B)
+        out, ref = run_both(agc, torch, G, code, p, bits, B, 4242, 9, masks)
+        assert_exact(out, ref)
+        return
+    rp, ci, a, w = _codes.identity_code(n)
+    w = (1.0 / (1.0 - p)).astype(np.float32)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=0, seed=17, flags=agc.AGC_FLAG_ALLOW_1BIT)
+    Gd = torch.zeros((k, (d + 3) // 4 * 4), dtype=torch.float32, device="cuda")
+    Gd[:, :d] = torch.from_numpy(G)
+    ses.encode(Gd, 2)
+    ghat = torch.full((R, d), -3.0, dtype=torch.float32, device="cuda")
+    ses.decode(torch.from_numpy(masks).cuda(), ghat=ghat)
+    torch.cuda.synchronize()
+    oc, osc, st, _ = orp.encode_quantize_global(rp, ci, a, bits, 17, 2, G)
+    og, _ = orp.decode(d, bits, 512, w, masks, oc, orp.expand_global_scales(osc, d))
+    assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
+    ses.close()
+
+
 @pytest.mark.parametrize("kind", ["cyclic", "interval"])
 def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch, kind):
     """Lemma 1 as a measured experiment: 20 rounds x 64 straggler realisations through the CUDA
