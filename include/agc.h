@@ -174,10 +174,11 @@ int agc_encode_quantize_rows(agc_plan_t *plan, const float *const *G_rows_dev, u
  * order with fused multiply-adds (reproducible bit for bit). With R > 1 and only
  * beta_dev the R updates are applied in one pass through the linear form
  * beta -= sum_i (sum_r lr_r I_{r,i}) w_i q_i, equal to the sequential updates up
- * to fp32 rounding. At least one of ghat_dev / beta_dev must be given. With only
+ * to fp32 rounding. At least one of ghat_dev / beta_dev must be given. With
  * ghat_dev and R >= 8 the realisations are decoded 64 at a time in one pass over
- * the messages (each message unpacked once per 64 realisations), with the same
- * results bit for bit as R single calls.
+ * the messages (each message unpacked once per 64 realisations) and beta_dev, if
+ * given, is then updated from the stored rows in order: the same results bit for
+ * bit as R single calls.
  * Asynchronous on the stream; R <= 4096.
  */
 int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,

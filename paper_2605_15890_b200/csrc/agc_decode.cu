@@ -856,6 +856,18 @@ __global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecPa
     }
 }
 
+// beta <- beta - lr_r * g_hat^(r) for r = 0..R-1 in order, from stored g_hat rows: the same fma
+// chain per coordinate as the fused update of realisation-by-realisation launches.
+__global__ void __launch_bounds__(256) agc_apply_updates_kernel(const float *ghat, const float *lr, int R, long long d,
+                                                                float *beta)
+{
+    for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < d; m += (long long)gridDim.x * blockDim.x) {
+        float b = beta[m];
+        for (int r = 0; r < R; ++r) b = __fmaf_rn(-__ldg(lr + r), __ldg(ghat + (long long)r * d + m), b);
+        beta[m] = b;
+    }
+}
+
 // Shared memory of the kernel above for RG groups of 16 realisations and n workers.
 size_t multi_smem_bytes(int rg, int rows_per_bucket, int n)
 {
@@ -977,11 +989,16 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
                                                                                plan->d_weff);
         P.weff = plan->d_weff;
     }
-    if (plan->dec_ring && ghat && !beta && R >= AGC_DEC_MULTI_MIN_R &&
+    if (plan->dec_ring && ghat && R >= AGC_DEC_MULTI_MIN_R &&
         multi_smem_bytes(4, P.rows_per_bucket, plan->n) <= size_t(plan->smem_optin)) {
-        if (P.rows_per_bucket == 4) return launch_multi_rb<4>(P, plan->sm_count, plan->smem_optin, stream);
-        if (P.rows_per_bucket == 2) return launch_multi_rb<2>(P, plan->sm_count, plan->smem_optin, stream);
-        return launch_multi_rb<1>(P, plan->sm_count, plan->smem_optin, stream);
+        const int rc = P.rows_per_bucket == 4   ? launch_multi_rb<4>(P, plan->sm_count, plan->smem_optin, stream)
+                       : P.rows_per_bucket == 2 ? launch_multi_rb<2>(P, plan->sm_count, plan->smem_optin, stream)
+                                                : launch_multi_rb<1>(P, plan->sm_count, plan->smem_optin, stream);
+        if (rc != AGC_OK || !beta) return rc;
+        // the R updates in order, from the rows just written
+        const long long want = (plan->d + 255) / 256, cap = (long long)plan->sm_count * 8;
+        agc_apply_updates_kernel<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(ghat, plan->d_lr, R, plan->d, beta);
+        return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
     }
     if (plan->dec_ring) {
         P.qt = ring_tile_height(plan->nblk, plan->sm_count, AGC_DEC_QT);

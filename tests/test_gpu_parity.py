@@ -572,8 +572,13 @@ def test_g_hat_of_many_realisations_in_one_pass(agc, torch, R, B, d, n):
     G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-3, 2, (k, 1))).astype(np.float32)
     if B:
         code = _codes.cyclic_code(p, bits, k, min(3, k), B)
-        out, ref = run_both(agc, torch, G, code, p, bits, B, 4242, 9, masks)
+        lr = rng.uniform(1e-3, 1e-1, R).astype(np.float32)
+        beta0 = rng.standard_normal(d).astype(np.float32)
+        out, ref = run_both(agc, torch, G, code, p, bits, B, 4242, 9, masks, lr=lr, beta0=beta0)
         assert_exact(out, ref)
+        # with the parameters as well: the R updates in order, from the stored rows
+        assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
+        assert np.abs(out["beta_fused"] - ref["beta"]).max() / np.abs(ref["beta"]).max() <= 1e-5
         return
     rp, ci, a, w = _codes.identity_code(n)
     w = (1.0 / (1.0 - p)).astype(np.float32)
