@@ -554,7 +554,8 @@ def test_global_norm_two_pass_encode_and_decode(agc, torch, d, direct):
 
 
 @pytest.mark.parametrize("R,B,d,n", [(8, 512, 5000, 12), (16, 256, 70_001, 9), (17, 128, 1300, 40), (33, 512, 513, 70),
-                                     (64, 512, 200_000, 20), (65, 256, 4097, 33), (130, 128, 3, 5), (48, 0, 40_000, 6)])
+                                     (64, 512, 200_000, 20), (65, 256, 4097, 33), (130, 128, 3, 5), (48, 0, 40_000, 6),
+                                     (9, 512, 1500, 300), (8, 256, 600, 2048)])
 def test_g_hat_of_many_realisations_in_one_pass(agc, torch, R, B, d, n):
     """From 8 realisations on, g_hat of every realisation comes from one pass over the messages
     (chunks of 64 realisations). Every row must equal the oracle's realisation-by-realisation
