@@ -220,6 +220,27 @@ int agc_decode_two_track(agc_plan_t *plan, const void *codes_dev, const float *s
                          const agc_adam_t *adam, uint32_t *status_dev, void *cuda_stream);
 
 /*
+ * agc_decode_residuals - squared residuals of many straggler realisations against a
+ * reference, for measuring the error bounds of Lemma 1 and Lemma 2 (Sec. III, IV) at full
+ * size: sqerr[r] = || g_hat^(r) - g_ref ||_2^2 with g_hat^(r) = sum_i I_{r,i} w_i q_i as in
+ * agc_decode, without storing any g_hat (64 realisations per pass over the messages).
+ *
+ *   codes_dev, scales_dev  device, as written by agc_encode_quantize
+ *   masks_dev  device, R x n bytes, 1 = arrived
+ *   g_ref_dev  device, d fp32: the vector to compare with (the exact sum of the partial
+ *              gradients, say); read only
+ *   sqerr_dev  device out, R doubles, overwritten
+ * Every g_hat^(r) is formed exactly as agc_decode forms it (fp32, workers ascending); the
+ * differences, their squares and the sum over 128 coordinates are fp32, the rest of the sum
+ * is fp64 and accumulated with atomic additions, so the last bits of a result may differ
+ * from run to run. Returns AGC_ERR_STATE for plans that cannot use the staged decoder
+ * (more than 2048 workers, AGC_FLAG_FORCE_DIRECT). Asynchronous on the stream; R <= 4096.
+ */
+int agc_decode_residuals(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+                         const uint8_t *masks_dev, int R, const float *g_ref_dev, double *sqerr_dev,
+                         void *cuda_stream);
+
+/*
  * agc_two_track_vector - the second-moment decoder of Sec. V-E in closed form:
  *   v_i = k Lambda / ((p_i + eta phi(b_i)) (sum_j a_ij) (1 + Lambda sum_m c_m^-1)),
  * c_m = (p_m + eta phi(b_m)) / (1 - p_m), k partitions, phi as in agc_bit_allocate.

@@ -69,6 +69,8 @@ def _load():
     L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
                                            vp, vp]
     L.agc_decode_update_static.restype = C.c_int
+    L.agc_decode_residuals.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp, vp]
+    L.agc_decode_residuals.restype = C.c_int
     L.agc_decode_two_track.argtypes = [vp, vp, vp, vp, f32p, vp, vp, vp, vp, vp, C.POINTER(AgcAdam), vp, vp]
     L.agc_decode_two_track.restype = C.c_int
     L.agc_two_track_vector.argtypes = [C.c_int, C.c_int, f64p, u8p, C.c_double, C.c_double, C.c_double, i32p, f32p,
@@ -193,6 +195,12 @@ def agc_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host=None, ghat_dev
     _check(_lib.agc_decode(plan, _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
                            _hp(lr, C.c_float), _dev(ghat_dev), _dev(beta_dev), _dev(status_dev),
                            _stream(stream)))
+
+
+def agc_decode_residuals(plan, codes_dev, scales_dev, masks_dev, R, g_ref_dev, sqerr_dev, stream=None):
+    """sqerr_dev: device float64 [R], overwritten with ||g_hat^(r) - g_ref||^2."""
+    _check(_lib.agc_decode_residuals(plan, _dev(codes_dev), _dev(scales_dev), _dev(masks_dev), R,
+                                     _dev(g_ref_dev), _dev(sqerr_dev), _stream(stream)))
 
 
 def agc_decode_update_static(n_workers, d, bucket, bits, w, codes_dev, scales_dev, masks_dev, R, lr_host,

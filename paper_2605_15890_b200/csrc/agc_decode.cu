@@ -693,7 +693,10 @@ __device__ __forceinline__ void multi_levels(const uint32_t (&W)[4], int lane, f
     }
 }
 
-template <int RB>
+// RES: instead of storing g_hat^(r), add ||g_hat^(r) - g_ref||^2 to sqerr[r] (squares and the sum
+// over a warp's 128 coordinates in fp32, everything above in fp64; lane j of a warp keeps the
+// running total of its j-th realisation and adds it to the output once, at the end).
+template <int RB, bool RES = false>
 __global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecParams P, int r0, int Rc)
 {
     extern __shared__ __align__(16) unsigned char multi_smem[];
@@ -771,6 +774,7 @@ __global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecPa
         }
     };
 
+    double res_total = 0.0;   // RES: lane j, realisation 16 rg + j
     prefetch(blockIdx.x, 0);
     int it = 0;   // batches so far: consecutive batches alternate between the two buffers, across blocks too
     for (long long q = blockIdx.x; q < P.nblk; q += gridDim.x) {
@@ -834,25 +838,49 @@ __global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecPa
         }
         // realisations 16 rg .. 16 rg + 15 of the chunk, coordinates 128 row + 4 lane .. + 3 of block q
         const long long m0 = q * AGC_BLOCK + 128 * row + 4 * lane;
+        if constexpr (RES) {
+            float g[4];
 #pragma unroll
-        for (int pr = 0; pr < 8; ++pr) {
+            for (int e = 0; e < 4; ++e) g[e] = m0 + e < P.d ? __ldg(P.gref + m0 + e) : 0.0f;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int r = 16 * rg + 2 * pr + h;
-                if (r >= Rc) continue;
-                float *out = P.ghat + (long long)(r0 + r) * P.d + m0;
-                const float v0 = h ? acc[pr][0].y : acc[pr][0].x, v1 = h ? acc[pr][1].y : acc[pr][1].x;
-                const float v2 = h ? acc[pr][2].y : acc[pr][2].x, v3 = h ? acc[pr][3].y : acc[pr][3].x;
-                if (vec && m0 + 3 < P.d) {
-                    *reinterpret_cast<float4 *>(out) = make_float4(v0, v1, v2, v3);
-                } else {
-                    if (m0 < P.d) out[0] = v0;
-                    if (m0 + 1 < P.d) out[1] = v1;
-                    if (m0 + 2 < P.d) out[2] = v2;
-                    if (m0 + 3 < P.d) out[3] = v3;
+            for (int pr = 0; pr < 8; ++pr) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float s = 0.0f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float diff = m0 + e < P.d ? __fsub_rn(h ? acc[pr][e].y : acc[pr][e].x, g[e]) : 0.0f;
+                        s = __fmaf_rn(diff, diff, s);
+                    }
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, off));
+                    if (lane == 2 * pr + h) res_total += (double)s;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int pr = 0; pr < 8; ++pr) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int r = 16 * rg + 2 * pr + h;
+                    if (r >= Rc) continue;
+                    float *out = P.ghat + (long long)(r0 + r) * P.d + m0;
+                    const float v0 = h ? acc[pr][0].y : acc[pr][0].x, v1 = h ? acc[pr][1].y : acc[pr][1].x;
+                    const float v2 = h ? acc[pr][2].y : acc[pr][2].x, v3 = h ? acc[pr][3].y : acc[pr][3].x;
+                    if (vec && m0 + 3 < P.d) {
+                        *reinterpret_cast<float4 *>(out) = make_float4(v0, v1, v2, v3);
+                    } else {
+                        if (m0 < P.d) out[0] = v0;
+                        if (m0 + 1 < P.d) out[1] = v1;
+                        if (m0 + 2 < P.d) out[2] = v2;
+                        if (m0 + 3 < P.d) out[3] = v3;
+                    }
                 }
             }
         }
+    }
+    if constexpr (RES) {
+        if (lane < 16 && 16 * rg + lane < Rc) atomicAdd(P.sqerr + r0 + 16 * rg + lane, res_total);
     }
 }
 
@@ -922,7 +950,7 @@ int ring_tile_height(long long nblk, int sm_count, int qt_max)
 }
 
 // g_hat of R >= AGC_DEC_MULTI_MIN_R realisations: chunks of up to 64 realisations per launch.
-template <int RB>
+template <int RB, bool RES = false>
 int launch_multi_rb(const AgcDecParams &P, int sm_count, int smem_optin, cudaStream_t stream)
 {
     for (int r0 = 0; r0 < P.R; r0 += 64) {
@@ -932,12 +960,12 @@ int launch_multi_rb(const AgcDecParams &P, int sm_count, int smem_optin, cudaStr
         const size_t smem = multi_smem_bytes(rg, RB, P.n);
         if (smem > size_t(smem_optin)) return AGC_ERR_STATE;
         int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agc_decode_multi_kernel<RB>, threads, smem) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agc_decode_multi_kernel<RB, RES>, threads, smem) != cudaSuccess ||
             per_sm < 1)
             return AGC_ERR_CUDA;
         const long long slots = (long long)sm_count * per_sm;
         const int grid = (int)(P.nblk < slots ? P.nblk : slots);
-        agc_decode_multi_kernel<RB><<<grid, threads, smem, stream>>>(P, r0, Rc);
+        agc_decode_multi_kernel<RB, RES><<<grid, threads, smem, stream>>>(P, r0, Rc);
         if (cudaGetLastError() != cudaSuccess) return AGC_ERR_CUDA;
     }
     return AGC_OK;
@@ -1023,6 +1051,39 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
 }
 
+// ||g_hat^(r) - g_ref||^2 of R realisations without storing any g_hat (sqerr: R doubles, overwritten).
+int agc_launch_decode_residuals(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks, int R,
+                                const float *g_ref, double *sqerr, cudaStream_t stream)
+{
+    if (!plan->dec_ring || multi_smem_bytes(4, plan->bucket / 128, plan->n) > size_t(plan->smem_optin))
+        return AGC_ERR_STATE;
+    AgcDecParams P;
+    P.bits = plan->d_bits;
+    P.w = plan->d_w;
+    P.word_off = plan->d_word_off;
+    P.codes = static_cast<const uint32_t *>(codes);
+    P.scales = scales;
+    P.masks = masks;
+    P.weff = nullptr;
+    P.ghat = nullptr;
+    P.beta = nullptr;
+    P.d = plan->d;
+    P.nblk = plan->nblk;
+    P.nb = plan->nb;
+    P.n = plan->n;
+    P.R = R;
+    P.rows_per_bucket = plan->bucket / 128;
+    P.global_norm = plan->global_norm ? 1 : 0;
+    P.lr0 = 0.0f;
+    P.lr = nullptr;
+    P.gref = g_ref;
+    P.sqerr = sqerr;
+    if (cudaMemsetAsync(sqerr, 0, sizeof(double) * R, stream) != cudaSuccess) return AGC_ERR_CUDA;
+    if (P.rows_per_bucket == 4) return launch_multi_rb<4, true>(P, plan->sm_count, plan->smem_optin, stream);
+    if (P.rows_per_bucket == 2) return launch_multi_rb<2, true>(P, plan->sm_count, plan->smem_optin, stream);
+    return launch_multi_rb<1, true>(P, plan->sm_count, plan->smem_optin, stream);
+}
+
 // Decide whether the plan decodes with the ring kernels and size their shared memory.
 int agc_decode_prepare(agc_plan *plan, int smem_optin)
 {
@@ -1036,7 +1097,10 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
         return AGC_ERR_CUDA;
     if (cudaFuncSetAttribute(agc_decode_multi_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
         cudaFuncSetAttribute(agc_decode_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
-        cudaFuncSetAttribute(agc_decode_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
+        cudaFuncSetAttribute(agc_decode_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_multi_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_multi_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_multi_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
         return AGC_ERR_CUDA;
     plan->smem_optin = smem_optin;
     plan->dec_ring = true;

@@ -106,6 +106,9 @@ struct AgcDecParams {
     int stages = 0;              // ring depth of the ring kernel
     int qt = 1;                  // blocks per tile of this ring launch (at most the kernel's QT)
     uint32_t w2_offset = 0;      // byte offset of the second-decoder array in shared memory
+    // residuals of many realisations
+    const float *gref = nullptr;  // d reference values
+    double *sqerr = nullptr;      // R sums of squared differences
     // two-track decode
     const float *v = nullptr;    // n second decoding coefficients
     float *ghat_v = nullptr;     // d or NULL
@@ -168,6 +171,8 @@ int agc_launch_encode(agc_plan *plan, const float *G, const float *const *G_rows
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
                       int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
                       cudaStream_t stream);
+int agc_launch_decode_residuals(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks, int R,
+                                const float *g_ref, double *sqerr, cudaStream_t stream);
 int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *scales, const uint8_t *mask,
                                 const float *v_host, float *ghat_w, float *ghat_v, float *beta, float *m,
                                 float *u, const agc_adam_t *adam, uint32_t *status, cudaStream_t stream);

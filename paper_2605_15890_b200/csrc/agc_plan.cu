@@ -318,6 +318,18 @@ extern "C" int agc_decode(agc_plan_t *plan, const void *codes_dev, const float *
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+extern "C" int agc_decode_residuals(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
+                                    const uint8_t *masks_dev, int R, const float *g_ref_dev, double *sqerr_dev,
+                                    void *cuda_stream)
+{
+    if (!plan || !codes_dev || !scales_dev || !masks_dev || !g_ref_dev || !sqerr_dev) return AGC_ERR_ARG;
+    if (R < 1) return AGC_ERR_ARG;
+    if (R > AGC_MAX_R) return AGC_ERR_STATE;
+    if (reinterpret_cast<uintptr_t>(codes_dev) & 15) return AGC_ERR_ALIGN;
+    return agc_launch_decode_residuals(plan, codes_dev, scales_dev, masks_dev, R, g_ref_dev, sqerr_dev,
+                                       static_cast<cudaStream_t>(cuda_stream));
+}
+
 extern "C" int agc_decode_two_track(agc_plan_t *plan, const void *codes_dev, const float *scales_dev,
                                     const uint8_t *mask_dev, const float *v_host, float *ghat_w_dev,
                                     float *ghat_v_dev, float *beta_dev, float *m_dev, float *u_dev,

@@ -51,6 +51,15 @@ class Session:
         R = masks.shape[0] if masks.dim() == 2 else 1
         B.agc_decode(self.plan, self.codes, self.scales, masks, R, lr, ghat, beta, self.status, stream)
 
+    def residuals(self, masks, g_ref, stream=None):
+        """||g_hat^(r) - g_ref||^2 of every realisation: float64 CUDA tensor [R]; no g_hat is stored."""
+        assert masks.dtype == torch.uint8 and masks.is_cuda and masks.is_contiguous()
+        assert g_ref.dtype == torch.float32 and g_ref.is_cuda and g_ref.is_contiguous() and g_ref.numel() == self.d
+        R = masks.shape[0] if masks.dim() == 2 else 1
+        out = torch.empty(R, dtype=torch.float64, device=masks.device)
+        B.agc_decode_residuals(self.plan, self.codes, self.scales, masks, R, g_ref, out, stream)
+        return out
+
     def worker_words(self, i):
         lo = B.agc_worker_offset(self.plan, i) // 4
         hi = B.agc_worker_offset(self.plan, i + 1) // 4

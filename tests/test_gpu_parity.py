@@ -596,6 +596,43 @@ def test_g_hat_of_many_realisations_in_one_pass(agc, torch, R, B, d, n):
     ses.close()
 
 
+@pytest.mark.parametrize("R,B,d,n", [(1, 512, 5000, 12), (20, 256, 70_001, 9), (64, 128, 200_000, 20), (70, 0, 40_000, 6)])
+def test_residuals_of_many_realisations_without_storing_g_hat(agc, torch, R, B, d, n):
+    """||g_hat^(r) - g||^2 for every realisation straight from the messages: against the oracle's
+    g_hat rows (fp32, defining order), differences squared and summed in fp64 on the host. The
+    library sums 128 coordinates in fp32 before it goes to fp64: 1e-6 relative."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(R * 77 + n)
+    k = n
+    bits = rng.integers(1, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.6, n)
+    masks = (rng.random((R, n)) >= p).astype(np.uint8)
+    masks[R // 2] = 0
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 1, (k, 1))).astype(np.float32)
+    g_ref = G.astype(np.float64).sum(0).astype(np.float32)
+    if B:
+        rp, ci, a, w = _codes.cyclic_code(p, bits, k, min(3, k), B)
+    else:
+        rp, ci, a, w = _codes.identity_code(n)
+        w = (1.0 / (1.0 - p)).astype(np.float32)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=5, flags=agc.AGC_FLAG_ALLOW_1BIT)
+    Gd = torch.zeros((k, (d + 3) // 4 * 4), dtype=torch.float32, device="cuda")
+    Gd[:, :d] = torch.from_numpy(G)
+    ses.encode(Gd, 3)
+    got = ses.residuals(torch.from_numpy(masks).cuda(), torch.from_numpy(g_ref).cuda()).cpu().numpy()
+    ses.close()
+    if B:
+        oc, osc, _, _ = orp.encode_quantize(rp, ci, a, bits, B, 5, 3, G, d=d)
+        og, _ = orp.decode(d, bits, B, w, masks, oc, osc)
+    else:
+        oc, osc, _, _ = orp.encode_quantize_global(rp, ci, a, bits, 5, 3, G)
+        og, _ = orp.decode(d, bits, 512, w, masks, oc, orp.expand_global_scales(osc, d))
+    want = ((og.astype(np.float64) - g_ref.astype(np.float64)[None]) ** 2).sum(1)
+    assert want[R // 2] == pytest.approx(float((g_ref.astype(np.float64) ** 2).sum()), rel=1e-12)   # nobody arrived
+    assert np.abs(got - want).max() <= 1e-6 * want.max()
+    assert (np.abs(got - want) <= 1e-6 * want).all()
+
+
 @pytest.mark.parametrize("kind", ["cyclic", "interval"])
 def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch, kind):
     """Lemma 1 as a measured experiment: 20 rounds x 64 straggler realisations through the CUDA
@@ -644,6 +681,39 @@ def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch, kind):
     # below the error of a single estimate
     assert np.linalg.norm(mean - g) <= 3.0 * np.sqrt(mse / rounds)
     assert np.linalg.norm(mean - g) <= 0.3 * np.sqrt(mse)
+    ses.close()
+
+
+def test_lemma1_bound_at_full_size_from_residuals(agc, torch):
+    """Lemma 1 measured at the size of the third configuration (n = k = 32, cyclic s = 4,
+    d = 25,557,032): 3 rounds x 64 straggler realisations, squared residuals reduced on the
+    device (no g_hat is stored). Their mean stays below the bound
+    C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 (||g_j||^2 = C = 1) and is not far below."""
+    from paper_2605_15890_b200.session import Session
+    wl = cfgs.config3()
+    B = 512
+    bits = np.array([8] * 10 + [6] + [2] * 21, np.uint8)
+    rp, ci, a, w = _codes.cyclic_code(wl.p, bits, wl.k, wl.s, B)
+    A = od.csr_to_dense(rp, ci, a.astype(np.float64), wl.k)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    G = torch.randn((wl.k, wl.d), generator=gen, device="cuda", dtype=torch.float32)
+    G /= G.double().pow(2).sum(1, keepdim=True).sqrt().float()                     # C = 1
+    g_ref = torch.zeros(wl.d, dtype=torch.float64, device="cuda")
+    for j in range(wl.k):
+        g_ref += G[j].double()
+    g_ref = g_ref.float()
+    ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, bits, bucket=B, seed=11)
+    rng = np.random.default_rng(12)
+    rounds, R = 3, 64
+    total = 0.0
+    for t in range(rounds):
+        masks = (rng.random((R, wl.n)) >= wl.p).astype(np.uint8)
+        ses.encode(G, t)
+        total += float(ses.residuals(torch.from_numpy(masks).cuda(), g_ref).sum().item())
+    assert int(ses.status.item()) == 0
+    mse = total / (rounds * R)
+    bound = od.lemma1_bound(A, w.astype(np.float64), wl.p, bits, B, C=1.0)
+    assert 0.05 * bound <= mse <= 1.05 * bound
     ses.close()
 
 
