@@ -688,7 +688,10 @@ def test_lemma1_bound_at_full_size_from_residuals(agc, torch):
     """Lemma 1 measured at the size of the third configuration (n = k = 32, cyclic s = 4,
     d = 25,557,032): 3 rounds x 64 straggler realisations, squared residuals reduced on the
     device (no g_hat is stored). Their mean stays below the bound
-    C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 (||g_j||^2 = C = 1) and is not far below."""
+    C sum_i (1-p_i){p_i + phi(b_i)} w_i^2 (sum_j a_ij)^2 (||g_j||^2 = C = 1), which is loose for
+    nearly orthogonal g_j, and not below the part of the error that stragglers alone cause,
+    sum_i p_i (1-p_i) w_i^2 ||f_i||^2 (the estimate is unbiased and the workers independent, so
+    the rounding noise only adds to it)."""
     from paper_2605_15890_b200.session import Session
     wl = cfgs.config3()
     B = 512
@@ -713,7 +716,14 @@ def test_lemma1_bound_at_full_size_from_residuals(agc, torch):
     assert int(ses.status.item()) == 0
     mse = total / (rounds * R)
     bound = od.lemma1_bound(A, w.astype(np.float64), wl.p, bits, B, C=1.0)
-    assert 0.05 * bound <= mse <= 1.05 * bound
+    assert mse <= 1.05 * bound
+    straggler_part = 0.0
+    for i in range(wl.n):
+        f = torch.zeros(wl.d, dtype=torch.float32, device="cuda")
+        for e in range(rp[i], rp[i + 1]):
+            f += float(a[e]) * G[int(ci[e])]
+        straggler_part += float(wl.p[i] * (1 - wl.p[i])) * float(w[i]) ** 2 * float(f.double().pow(2).sum().item())
+    assert straggler_part > 0 and mse >= 0.6 * straggler_part    # 192 realisations: the sample mean is within tens of per cent
     ses.close()
 
 
