@@ -29,14 +29,55 @@ __device__ __forceinline__ T load_words(const T *p)
     else return *p;
 }
 
+// Words of a lane's 16 codes: (16 BITS + 31) / 32 of them, plus a zero word for the extraction
+// of a code that would straddle the end.
+template <int BITS>
+struct LaneWords {
+    static constexpr int NACC = (16 * BITS + 31) / 32;
+    uint32_t A[NACC + 1];
+};
+
+// Odd widths: a pair of lanes shares BITS words and the odd lane's slice starts at bit 16 of
+// word H = (BITS - 1) / 2. From the H + 1 words a lane reads (the even lane from word 0, the
+// odd lane from word H) to its own slice.
+template <int BITS>
+__device__ __forceinline__ void odd_width_slice(const uint32_t *W, int lane, LaneWords<BITS> &out)
+{
+    constexpr int H = (BITS - 1) / 2;
+    if (lane & 1) {
+#pragma unroll
+        for (int t = 0; t < H; ++t) out.A[t] = __funnelshift_r(W[t], W[t + 1], 16);
+        out.A[H] = W[H] >> 16;
+    } else {
+#pragma unroll
+        for (int t = 0; t <= H; ++t) out.A[t] = W[t];
+    }
+}
+
+// Level t of the lane (code - L, or code - 1/2 for one-bit codes), exact in fp32.
+template <int BITS>
+__device__ __forceinline__ float level_of(const LaneWords<BITS> &lw, int t)
+{
+    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+    const int bitpos = t * BITS;
+    const int w = bitpos >> 5, sh = bitpos & 31;
+    uint32_t code;
+    if (sh + BITS <= 32) code = (lw.A[w] >> sh) & MASK;
+    else code = __funnelshift_r(lw.A[w], lw.A[w + 1], sh) & MASK;
+    if constexpr (BITS >= 2)
+        return __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);  // code - L, exact
+    else
+        return __uint_as_float(0xBF000000u ^ (code << 31));                          // code - 0.5
+}
+
 template <int BITS, bool GLOBAL = true>
 __device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int lane,
                                                   const float (&cstep_row)[4], float (&acc)[16])
 {
-    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS - 1)) - 1u : 0u;
-    constexpr uint32_t MASK = (1u << BITS) - 1u;
-    constexpr int NACC = (16 * BITS + 31) / 32;
-    uint32_t A[NACC + 1];
+    constexpr int NACC = LaneWords<BITS>::NACC;
+    LaneWords<BITS> lw;
+    uint32_t (&A)[NACC + 1] = lw.A;
     A[NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
         constexpr int NW = BITS / 2;
@@ -58,29 +99,10 @@ __device__ __forceinline__ void unpack_accumulate(const uint32_t *blk_words, int
         uint32_t W[H + 1];
 #pragma unroll
         for (int t = 0; t <= H; ++t) W[t] = load_words<GLOBAL>(src + t);
-        if (lane & 1) {
-#pragma unroll
-            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
-            A[H] = W[H] >> 16;
-        } else {
-#pragma unroll
-            for (int t = 0; t <= H; ++t) A[t] = W[t];
-        }
+        odd_width_slice<BITS>(W, lane, lw);
     }
 #pragma unroll
-    for (int t = 0; t < 16; ++t) {
-        const int bitpos = t * BITS;
-        const int w = bitpos >> 5, sh = bitpos & 31;
-        uint32_t code;
-        if (sh + BITS <= 32) code = (A[w] >> sh) & MASK;
-        else code = __funnelshift_r(A[w], A[w + 1], sh) & MASK;
-        float level;
-        if constexpr (BITS >= 2)
-            level = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);  // code - L, exact
-        else
-            level = __uint_as_float(0xBF000000u ^ (code << 31));                          // code - 0.5
-        acc[t] = __fmaf_rn(cstep_row[t >> 2], level, acc[t]);
-    }
+    for (int t = 0; t < 16; ++t) acc[t] = __fmaf_rn(cstep_row[t >> 2], level_of<BITS>(lw, t), acc[t]);
 }
 
 template <int RB>
@@ -255,14 +277,15 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
     constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
     constexpr uint32_t MASK = (1u << BITS) - 1u;
     constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)(BITS >= 2 ? L : 1u)) : 2.0f;
-    constexpr int NACC = (16 * BITS + 31) / 32;
+    constexpr int NACC = LaneWords<BITS>::NACC;
     float cstep_row[4], cstep2_row[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
         cstep2_row[c] = TWO ? __fmul_rn(ws2_row[c], DSTEP) : 0.0f;
     }
-    uint32_t A[NACC + 1];
+    LaneWords<BITS> lw;
+    uint32_t (&A)[NACC + 1] = lw.A;
     A[NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
         constexpr int NW = BITS / 2;
@@ -283,14 +306,7 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
         uint32_t W[H + 1];
 #pragma unroll
         for (int t = 0; t <= H; ++t) W[t] = lds32(src + 4 * t);
-        if (lane & 1) {
-#pragma unroll
-            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
-            A[H] = W[H] >> 16;
-        } else {
-#pragma unroll
-            for (int t = 0; t <= H; ++t) A[t] = W[t];
-        }
+        odd_width_slice<BITS>(W, lane, lw);
     }
     // two coordinates at a time: the subtraction and the fma are packed instructions (two
     // independent IEEE fp32 operations each), which halves their issue slots
@@ -656,41 +672,21 @@ struct __align__(16) AgcMultiWorker {
     int pad;
 };
 
-// The lane's 16 levels (code - L, or code - 1/2 for one-bit codes) from its words of the block.
+// The lane's 16 levels from the words it fetched ahead (even widths: its own BITS / 2 words; odd
+// widths: the H + 1 words of odd_width_slice).
 template <int BITS>
 __device__ __forceinline__ void multi_levels(const uint32_t (&W)[4], int lane, float (&lv)[16])
 {
-    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
-    constexpr uint32_t MASK = (1u << BITS) - 1u;
-    constexpr int NACC = (16 * BITS + 31) / 32;
-    uint32_t A[NACC + 1];
-    A[NACC] = 0u;
+    LaneWords<BITS> lw;
+    lw.A[LaneWords<BITS>::NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
 #pragma unroll
-        for (int t = 0; t < NACC; ++t) A[t] = W[t];
+        for (int t = 0; t < LaneWords<BITS>::NACC; ++t) lw.A[t] = W[t];
     } else {
-        constexpr int H = (BITS - 1) / 2;
-        if (lane & 1) {
-#pragma unroll
-            for (int t = 0; t < H; ++t) A[t] = __funnelshift_r(W[t], W[t + 1], 16);
-            A[H] = W[H] >> 16;
-        } else {
-#pragma unroll
-            for (int t = 0; t <= H; ++t) A[t] = W[t];
-        }
+        odd_width_slice<BITS>(W, lane, lw);
     }
 #pragma unroll
-    for (int t = 0; t < 16; ++t) {
-        const int bitpos = t * BITS;
-        const int w = bitpos >> 5, sh = bitpos & 31;
-        uint32_t code;
-        if (sh + BITS <= 32) code = (A[w] >> sh) & MASK;
-        else code = __funnelshift_r(A[w], A[w + 1], sh) & MASK;
-        if constexpr (BITS >= 2)
-            lv[t] = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);  // code - L, exact
-        else
-            lv[t] = __uint_as_float(0xBF000000u ^ (code << 31));                          // code - 0.5
-    }
+    for (int t = 0; t < 16; ++t) lv[t] = level_of<BITS>(lw, t);
 }
 
 // RES: instead of storing g_hat^(r), add ||g_hat^(r) - g_ref||^2 to sqerr[r] (squares and the sum
