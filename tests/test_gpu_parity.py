@@ -727,6 +727,62 @@ def test_lemma1_bound_at_full_size_from_residuals(agc, torch):
     ses.close()
 
 
+@pytest.mark.parametrize("n,d,B", [(4, 10_000, 512), (64, 4096, 256), (6, 40_000, 0)])
+def test_rounds_captured_in_a_cuda_graph_replay_bit_for_bit(agc, torch, n, d, B):
+    """Small problems are bound by launch latency, so a caller may record several rounds
+    (encode + fused update each) in a CUDA graph: the entry points allocate nothing, copy nothing
+    from the host for one realisation and synchronise nothing. A replay must give the bits of the
+    same calls made one by one."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(n + d)
+    k = n
+    bits = rng.integers(2, 9, n).astype(np.uint8)
+    p = rng.uniform(0.05, 0.4, n)
+    if B:
+        rp, ci, a, w = _codes.cyclic_code(p, bits, k, 2, B)
+    else:
+        rp, ci, a, w = _codes.identity_code(n)
+        w = (1.0 / (1.0 - p)).astype(np.float32)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=3)
+    G = torch.from_numpy(rng.standard_normal((k, d)).astype(np.float32)).cuda()
+    mask = torch.from_numpy((rng.random(n) >= p).astype(np.uint8)).cuda()
+    lr = np.array([1e-2], np.float32)
+    beta0 = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).cuda()
+    rounds = 4
+
+    def run_rounds(beta):
+        for t in range(rounds):
+            ses.encode(G, t)
+            ses.decode(mask, lr=lr, beta=beta)
+
+    eager = beta0.clone()
+    run_rounds(eager)
+    codes_eager = ses.codes.clone()
+    torch.cuda.synchronize()
+    beta = beta0.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run_rounds(beta)                      # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    beta.copy_(beta0)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        run_rounds(beta)
+    beta.copy_(beta0)
+    ses.codes.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(beta.view(torch.int32), eager.view(torch.int32))
+    assert torch.equal(ses.codes, codes_eager)
+    run_rounds(eager)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(beta.view(torch.int32), eager.view(torch.int32))
+    assert int(ses.status.item()) == 0
+    ses.close()
+
+
 @pytest.mark.parametrize("d,B", [(1, 128), (513, 256), (70_001, 512), (40_000, 0)])
 def test_kernels_write_nothing_outside_their_outputs(agc, torch, d, B):
     """Guard words before and after every output buffer (messages, scales, g_hat, parameters,
