@@ -783,6 +783,44 @@ def test_rounds_captured_in_a_cuda_graph_replay_bit_for_bit(agc, torch, n, d, B)
     ses.close()
 
 
+def test_decode_entry_points_reject_bad_arguments(agc, torch):
+    """Error codes instead of launches: missing buffers, R out of range, misaligned messages, and
+    the entry points that need the staged decoder on a plan that was told not to use it."""
+    from paper_2605_15890_b200.session import Session
+    n = k = 4
+    d = 3000
+    bits = np.array([2, 3, 4, 8], np.uint8)
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 2, 512)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=512, seed=1)
+    direct = Session(n, k, d, rp, ci, a, w, p, bits, bucket=512, seed=1, flags=agc.AGC_FLAG_FORCE_DIRECT)
+    mask = torch.ones(n, dtype=torch.uint8, device="cuda")
+    ghat = torch.zeros(d, dtype=torch.float32, device="cuda")
+    sq = torch.zeros(4, dtype=torch.float64, device="cuda")
+
+    def code_of(fn):
+        with pytest.raises(agc.AgcError) as e:
+            fn()
+        return e.value.code
+
+    ERR_ARG, ERR_ALIGN, ERR_STATE = -1, -4, -7
+    assert code_of(lambda: agc.agc_decode(ses.plan, ses.codes, ses.scales, mask, 1)) == ERR_ARG            # no output
+    assert code_of(lambda: agc.agc_decode(ses.plan, ses.codes, ses.scales, mask, 0, None, ghat)) == ERR_ARG
+    assert code_of(lambda: agc.agc_decode(ses.plan, ses.codes, ses.scales, mask, 1, None, None, ghat)) == ERR_ARG  # beta without lr
+    assert code_of(lambda: agc.agc_decode(ses.plan, ses.codes, ses.scales, mask, 5000, None, ghat)) == ERR_STATE
+    off = ses.codes.view(torch.uint8)[4:]
+    assert code_of(lambda: agc.agc_decode(ses.plan, off, ses.scales, mask, 1, None, ghat)) == ERR_ALIGN
+    assert code_of(lambda: agc.agc_decode_residuals(ses.plan, ses.codes, ses.scales, mask, 0, ghat, sq)) == ERR_ARG
+    assert code_of(lambda: agc.agc_decode_residuals(ses.plan, ses.codes, ses.scales, mask, 1, None, sq)) == ERR_ARG
+    assert code_of(lambda: agc.agc_decode_residuals(ses.plan, off, ses.scales, mask, 1, ghat, sq)) == ERR_ALIGN
+    assert code_of(lambda: agc.agc_decode_residuals(direct.plan, direct.codes, direct.scales, mask, 1, ghat, sq)) == ERR_STATE
+    assert code_of(lambda: agc.agc_decode_two_track(direct.plan, direct.codes, direct.scales, mask,
+                                                    np.ones(n, np.float32), ghat)) == ERR_STATE
+    torch.cuda.synchronize()
+    ses.close()
+    direct.close()
+
+
 @pytest.mark.parametrize("d,B", [(1, 128), (513, 256), (70_001, 512), (40_000, 0)])
 def test_kernels_write_nothing_outside_their_outputs(agc, torch, d, B):
     """Guard words before and after every output buffer (messages, scales, g_hat, parameters,
