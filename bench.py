@@ -409,7 +409,10 @@ def main():
                 "config": workload_config(wl, bits, bucket, l2_note),
                 "kernels": {"encode_quantize_ms": k1_ms, "decode_update_ms": k2_ms, "staged_tma": bool(ses.uses_tma),
                             "status_bits": status, "two_track_adam_ms": tt_ms,
-                            "decode_GBs": k2_algorithmic_bytes(wl, bits, bucket, masks_all, wl.p) / (k2_ms * 1e-3) / 1e9},
+                            "decode_GBs": k2_algorithmic_bytes(wl, bits, bucket, masks_all, wl.p) / (k2_ms * 1e-3) / 1e9,
+                            "encode_GBs": achieved,
+                            "encode_coords_per_s": wl.d / (k1_ms * 1e-3), "decode_coords_per_s": wl.d / (k2_ms * 1e-3),
+                            "worker_coords_per_s": world * wl.n * wl.d / (step_ms * 1e-3)},
                 "roofline": {"bound": "hbm", "kernel": "agc_encode_staged_kernel" if ses.uses_tma else "agc_encode_direct_kernel",
                              "achieved": achieved, "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
                              "frac": achieved / peak, "frac_of_8000": achieved / 8000.0,
@@ -417,7 +420,9 @@ def main():
                              "traffic": None if tpc is None else tpc * wl.d,
                              "issue": issue_rate(wl, bucket, k1_ms, clocks)},
                 "clocks": clocks, "e2e": e2e,
-                "gpu_launches": args.steps * (2 + (1 if R > 1 else 0))}
+                # encode (global norm: first pass, two reduction kernels, second pass), decode, and the
+                # effective-weights kernel of a multi-realisation update
+                "gpu_launches": args.steps * ((4 if bucket == 0 else 1) + 1 + (1 if R > 1 else 0))}
         if not args.no_cpu_baseline:
             rate, secs, d_s = oracle_sample_rate(wl, code, bits, bucket)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
