@@ -456,3 +456,83 @@ uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_
     free(x); free(part);
     return status;
 }
+
+/*
+ * Buckets of B = 1024, 2048 or 4096 coordinates (Sec. II-B calls the bucket-wise variant of
+ * Eq. quant_def straightforward; it fixes no bucket size). Such a bucket spans group = B / 512
+ * pack blocks. Its sum of squares is formed like the global one above, from the pack blocks'
+ * sums (each by the 512-coordinate rule) with the same pairwise tree in block order, cut at the
+ * bucket: bucket t of a worker covers blocks [t * group, (t + 1) * group) and a block without a
+ * partner (ragged end) counts as it is. group = 1 is the 512-bucket encoder, group >= number of
+ * blocks the global-norm encoder. scales: n x nb, nb = ceil(nblk / group).
+ */
+uint32_t agc_oracle_encode_quantize_grouped(int n, int k, int64_t d, const int32_t *row_ptr,
+                                            const int32_t *col_idx, const float *a,
+                                            const uint8_t *bits, int64_t group, uint64_t seed,
+                                            uint64_t round, const float *G, int64_t ld,
+                                            uint32_t *codes, float *scales, float *x_out)
+{
+    const int64_t nblk = agc_oracle_num_blocks(d);
+    const int64_t nb = (nblk + group - 1) / group;
+    uint32_t status = 0;
+    float *x = (float *)malloc((size_t)nblk * AGC_BLOCK * sizeof(float));
+    float *part = (float *)malloc((size_t)nblk * sizeof(float));
+    int64_t woff = 0;
+    (void)k;
+    for (int i = 0; i < n; ++i) {
+        const int b = bits[i];
+        /* Sec. II-A: f_i, ascending partitions, fp32 fma chain; zero beyond d */
+        for (int64_t m = 0; m < nblk * AGC_BLOCK; ++m) {
+            float acc = 0.0f;
+            if (m < d)
+                for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                    acc = fmaf(a[e], G[(int64_t)col_idx[e] * ld + m], acc);
+            x[m] = acc;
+        }
+        if (x_out) memcpy(x_out + (int64_t)i * d, x, (size_t)d * sizeof(float));
+        for (int64_t q = 0; q < nblk; ++q) part[q] = bucket_sumsq(x + q * AGC_BLOCK, AGC_BLOCK);
+        uint32_t *words = codes + woff;
+        memset(words, 0, (size_t)nblk * 16 * b * sizeof(uint32_t));
+        for (int64_t t = 0; t < nb; ++t) {
+            const int64_t q0 = t * group;
+            int64_t len = nblk - q0 < group ? nblk - q0 : group;
+            const int64_t q1 = q0 + len;
+            float *v = part + q0;
+            /* shrinking tree over the bucket's block sums */
+            while (len > 1) {
+                int64_t half = (len + 1) / 2;
+                for (int64_t u = 0; u < half; ++u)
+                    v[u] = v[2 * u] + (2 * u + 1 < len ? v[2 * u + 1] : 0.0f);
+                len = half;
+            }
+            float sumsq = v[0];
+            int finite = (sumsq == sumsq) && (sumsq != INFINITY);
+            int flushed = !(finite && sumsq >= 1.17549435e-38f);
+            if (!finite) status |= AGC_ORACLE_STATUS_NONFINITE;
+            float S = flushed ? 0.0f : sqrtf(sumsq);
+            scales[(int64_t)i * nb + t] = S;
+            float inv = flushed ? 0.0f : agc_oracle_inv_scale(S, b);
+            for (int64_t q = q0; q < q1; ++q)
+                for (int o = 0; o < AGC_BLOCK; ++o) {
+                    int pos = stream_pos_in_block(o);
+                    uint32_t code;
+                    if (flushed) {
+                        code = zero_code(b);
+                    } else {
+                        uint32_t u = agc_oracle_uniform15(seed, round, (uint32_t)i,
+                                                          (uint64_t)q * AGC_BLOCK + (uint64_t)pos);
+                        code = agc_oracle_quantize_one(x[q * AGC_BLOCK + o], inv, b, u);
+                        if (code > 2u * zero_code(b) + (b == 1 ? 1u : 0u)) status |= AGC_ORACLE_STATUS_RANGE;
+                        code &= (1u << b) - 1u;
+                    }
+                    int bit = pos * b;
+                    uint32_t *w = words + q * 16 * b;
+                    w[bit >> 5] |= code << (bit & 31);
+                    if ((bit & 31) + b > 32) w[(bit >> 5) + 1] |= code >> (32 - (bit & 31));
+                }
+        }
+        woff += nblk * 16 * b;
+    }
+    free(x); free(part);
+    return status;
+}

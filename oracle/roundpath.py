@@ -52,6 +52,9 @@ def lib():
         L.agc_oracle_encode_quantize_global.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_uint64,
                                                         C.c_uint64, f32p, C.c_int64, u32p, f32p, f32p]
         L.agc_oracle_encode_quantize_global.restype = C.c_uint32
+        L.agc_oracle_encode_quantize_grouped.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_int64,
+                                                         C.c_uint64, C.c_uint64, f32p, C.c_int64, u32p, f32p, f32p]
+        L.agc_oracle_encode_quantize_grouped.restype = C.c_uint32
         L.agc_oracle_adam_two_track.argtypes = [C.c_int64, f32p, f32p, C.c_float, C.c_float, C.c_float, C.c_float,
                                                 C.c_float, C.c_float, C.c_float, C.c_float, f32p, f32p, f32p]
         L.agc_oracle_adam_two_track.restype = None
@@ -237,6 +240,37 @@ def encode_quantize_global(row_ptr, col_idx, a, bits, seed, rnd, G, d=None, want
                                                  _p(G, C.c_float), ld, _p(codes, C.c_uint32),
                                                  _p(scales, C.c_float), _p(x, C.c_float))
     return codes, scales, int(st), x
+
+
+def encode_quantize_grouped(row_ptr, col_idx, a, bits, B, seed, rnd, G, d=None, want_x=False):
+    """Encode + quantise + pack with buckets of B = 1024, 2048 or 4096 coordinates (whole groups
+    of pack blocks). Returns (codes uint32, scales float32 [n, ceil(d / B)], status, x or None)."""
+    assert B % BLOCK == 0 and B >= BLOCK
+    G = np.asarray(G)
+    assert G.dtype == np.float32 and G.ndim == 2 and G.strides[1] == 4
+    k = G.shape[0]
+    d = G.shape[1] if d is None else d
+    ld = G.strides[0] // 4
+    row_ptr, col_idx = _c(row_ptr, np.int32), _c(col_idx, np.int32)
+    a, bits = _c(a, np.float32), _c(bits, np.uint8)
+    n = len(bits)
+    group = B // BLOCK
+    nb = (num_blocks(d) + group - 1) // group
+    off = worker_word_offsets(d, bits)
+    codes = np.zeros(int(off[-1]), np.uint32)
+    scales = np.zeros((n, nb), np.float32)
+    x = np.zeros((n, d), np.float32) if want_x else None
+    st = lib().agc_oracle_encode_quantize_grouped(n, k, d, _p(row_ptr, C.c_int32), _p(col_idx, C.c_int32),
+                                                  _p(a, C.c_float), _p(bits, C.c_uint8), group, seed, rnd,
+                                                  _p(G, C.c_float), ld, _p(codes, C.c_uint32),
+                                                  _p(scales, C.c_float), _p(x, C.c_float))
+    return codes, scales, int(st), x
+
+
+def expand_grouped_scales(scales, d, B):
+    """Scales of buckets of B >= 512 coordinates as an (n, nblk) array for decode() with B = 512."""
+    group = B // BLOCK
+    return np.ascontiguousarray(np.repeat(np.asarray(scales, np.float32), group, axis=1)[:, :num_blocks(d)])
 
 
 def expand_global_scales(scales, d):

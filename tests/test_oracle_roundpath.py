@@ -499,3 +499,75 @@ def test_global_norm_encoder_pins():
         L = (1 << (int(bits[i]) - 1)) - 1
         sigma = scales[i] / L / 2.0 / np.sqrt(rounds)       # per-coordinate std of the mean is at most this
         assert np.abs(acc[i] / rounds - x[i]).max() <= 6.0 * sigma
+
+
+def test_grouped_bucket_encoder_pins():
+    """Buckets of 1024 / 2048 / 4096 coordinates (whole groups of pack blocks), pinned from both
+    ends and from outside: (i) a group of one block is the 512-bucket encoder bit for bit;
+    (ii) a group that covers every block is the global-norm encoder bit for bit; (iii) every
+    bucket's scale equals the float64 l2 norm of that stretch of f_i to fp32 accuracy, a zero
+    stretch is sent as zero codes with scale 0, and every dequantised value lies within one
+    level step of its bucket; (iv) the bucket boundaries are where they should be: changing one
+    value changes the scale of its own bucket only; (v) E[Q(x)] = x by Monte-Carlo."""
+    rng = np.random.default_rng(33)
+    n = k = 4
+    bits = np.array([2, 3, 5, 8], np.uint8)
+    rp = np.arange(n + 1, dtype=np.int32)
+    ci = np.arange(n, dtype=np.int32)
+    a = np.ones(n, np.float32)
+    d = 512 * 9 + 77                                    # 10 pack blocks, the last one ragged
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 2, (k, 1))).astype(np.float32)
+    # (i)
+    c1, s1, st1, _ = orp.encode_quantize_grouped(rp, ci, a, bits, 512, 3, 5, G)
+    c2, s2, st2, _ = orp.encode_quantize(rp, ci, a, bits, 512, 3, 5, G)
+    assert st1 == 0 and st2 == 0 and (c1 == c2).all() and (s1.view(np.uint32) == s2.view(np.uint32)).all()
+    # (ii)
+    c1, s1, _, _ = orp.encode_quantize_grouped(rp, ci, a, bits, 512 * 16, 3, 5, G)
+    c2, s2, _, _ = orp.encode_quantize_global(rp, ci, a, bits, 3, 5, G)
+    assert s1.shape == (n, 1) and (c1 == c2).all() and (s1[:, 0].view(np.uint32) == s2.view(np.uint32)).all()
+    # (iii)
+    G[2, 2048:4096] = 0.0
+    for B in (1024, 2048, 4096):
+        codes, scales, st, x = orp.encode_quantize_grouped(rp, ci, a, bits, B, 3, 5, G, want_x=True)
+        nb = (d + B - 1) // B
+        assert st == 0 and scales.shape == (n, nb)
+        xp = np.zeros((n, nb * B))
+        xp[:, :d] = x
+        want = np.sqrt((xp.reshape(n, nb, B) ** 2).sum(axis=2))
+        assert np.allclose(scales, want, rtol=3e-6, atol=0)
+        per_block = orp.expand_grouped_scales(scales, d, B)
+        assert per_block.shape == (n, orp.num_blocks(d))
+        off = orp.worker_word_offsets(d, bits)
+        for i in range(n):
+            qi = orp.dequantize_worker(d, int(bits[i]), 512, codes[off[i]:off[i + 1]], per_block[i])
+            L = (1 << (int(bits[i]) - 1)) - 1
+            step = np.repeat(per_block[i], 512)[:d] / L
+            assert (np.abs(qi - x[i]) <= step * 1.0001).all()
+        t0 = 2048 // B
+        if B <= 2048:
+            assert (scales[2, t0:4096 // B] == 0.0).all()
+            assert (orp.dequantize_worker(d, int(bits[2]), 512, codes[off[2]:off[3]], per_block[2])[2048:4096] == 0).all()
+    # (iv)
+    for B in (1024, 2048):
+        _, s_a, _, _ = orp.encode_quantize_grouped(rp, ci, a, bits, B, 3, 5, G)
+        G2 = G.copy()
+        m = 3 * 1024 + 5
+        G2[1, m] += 100.0
+        _, s_b, _, _ = orp.encode_quantize_grouped(rp, ci, a, bits, B, 3, 5, G2)
+        changed = np.argwhere(s_a.view(np.uint32) != s_b.view(np.uint32))
+        assert changed.tolist() == [[1, m // B]]
+    # (v)
+    d = 1500
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    acc = np.zeros((n, d))
+    rounds = 1500
+    for t in range(rounds):
+        codes, scales, _, x = orp.encode_quantize_grouped(rp, ci, a, bits, 1024, 9, t, G, want_x=True)
+        off = orp.worker_word_offsets(d, bits)
+        per_block = orp.expand_grouped_scales(scales, d, 1024)
+        for i in range(n):
+            acc[i] += orp.dequantize_worker(d, int(bits[i]), 512, codes[off[i]:off[i + 1]], per_block[i])
+    for i in range(n):
+        L = (1 << (int(bits[i]) - 1)) - 1
+        sigma = np.repeat(per_block[i], 512)[:d] / L / 2.0 / np.sqrt(rounds)
+        assert (np.abs(acc[i] / rounds - x[i]) <= 6.0 * sigma + 1e-12).all()
