@@ -55,7 +55,8 @@ def k1_algorithmic_bytes(wl, bits, bucket):
     if bucket == 0:   # global norm: the partial gradients are read twice, one scale per worker
         return 8 * wl.k * wl.d + int(sum(4 * 16 * int(b) * nblk for b in bits)) + 4 * wl.n
     nb = (wl.d + bucket - 1) // bucket
-    return 4 * wl.k * wl.d + int(sum(4 * 16 * int(b) * nblk for b in bits)) + 4 * wl.n * nb
+    passes = 2 if bucket > 512 else 1   # buckets of several pack blocks: two passes as well
+    return 4 * passes * wl.k * wl.d + int(sum(4 * 16 * int(b) * nblk for b in bits)) + 4 * wl.n * nb
 
 
 def k2_algorithmic_bytes(wl, bits, bucket, masks_all, p):
@@ -130,7 +131,10 @@ class ClockSampler:
 def oracle_round(orp, code, bits, bucket, seed, t, G, d, mask, lr, beta):
     """One round of the oracle: encode + quantise + pack, then decode + update (returns beta)."""
     rp, ci, a, w = code
-    if bucket:
+    if bucket > 512:
+        c, s0, _, _ = orp.encode_quantize_grouped(rp, ci, a, bits, bucket, seed, t, G, d=d)
+        s, B = orp.expand_grouped_scales(s0, d, bucket), 512
+    elif bucket:
         c, s, _, _ = orp.encode_quantize(rp, ci, a, bits, bucket, seed, t, G, d=d)
         B = bucket
     else:
@@ -144,7 +148,7 @@ def parity_sample(ses, G, wl, code, bits, bucket, blocks=(0, 1, 2, 3)):
     """The messages the GPU produced for the bench's own inputs against the oracle on a few pack
     blocks (first ones and the last): counts of differing code words and scales (expected 0).
     Bucket-wise mode only (the global norm needs the whole vector)."""
-    if not bucket:
+    if not bucket or bucket > 512:
         return None
     from oracle import roundpath as orp
     rp, ci, a, w = code
@@ -270,7 +274,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
-    ap.add_argument("--bucket", type=int, default=512, help="128, 256, 512, or 0 = one norm per worker (two-pass encode)")
+    ap.add_argument("--bucket", type=int, default=512, help="128, 256, 512 (one pass), 1024, 2048, 4096 or 0 = one norm per worker (two-pass encode)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -420,9 +424,10 @@ def main():
                              "traffic": None if tpc is None else tpc * wl.d,
                              "issue": issue_rate(wl, bucket, k1_ms, clocks)},
                 "clocks": clocks, "e2e": e2e,
-                # encode (global norm: first pass, two reduction kernels, second pass), decode, and the
+                # encode (global norm: first pass, two reduction kernels, second pass; buckets of several
+                # pack blocks: first pass, one reduction kernel, second pass), decode, and the
                 # effective-weights kernel of a multi-realisation update
-                "gpu_launches": args.steps * ((4 if bucket == 0 else 1) + 1 + (1 if R > 1 else 0))}
+                "gpu_launches": args.steps * ((4 if bucket == 0 else 3 if bucket > 512 else 1) + 1 + (1 if R > 1 else 0))}
         if not args.no_cpu_baseline:
             rate, secs, d_s = oracle_sample_rate(wl, code, bits, bucket)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",

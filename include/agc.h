@@ -80,10 +80,13 @@ typedef struct agc_plan agc_plan_t;
  *   w          host, n entries: decoding coefficients w_i
  *   p          host, n entries: straggler probabilities, 0 <= p_i < 1
  *   bits       host, n entries: b_i in 2..8 (1 with AGC_FLAG_ALLOW_1BIT)
- *   bucket     coordinates per scale: 128, 256 or 512; 0 = ONE l2 norm per worker over all d
- *              coordinates, the main formulation of Sec. II-B (the encoder then reads the
- *              partial gradients twice: block sums of squares, their pairwise-tree
- *              reduction, rounding with the global norm; scales holds n entries)
+ *   bucket     coordinates per scale: 128, 256 or 512 (one pass over the partial gradients);
+ *              1024, 2048 or 4096 (buckets of 2, 4 or 8 blocks of 512 coordinates); 0 = ONE
+ *              l2 norm per worker over all d coordinates, the main formulation of Sec. II-B
+ *              (scales then holds n entries). For 1024 and above and for 0 the encoder reads
+ *              the partial gradients twice: sums of squares of the 512-coordinate blocks,
+ *              their pairwise-tree reduction in block order over the bucket (or over the whole
+ *              vector), then the rounding with the resulting norm
  *   seed       key of the counter-based random stream of the stochastic rounding
  *   flags      AGC_FLAG_*
  * All host arrays are copied. Unless AGC_FLAG_NO_UNBIASED_CHECK is set the
@@ -115,7 +118,8 @@ size_t agc_worker_offset(const agc_plan_t *plan, int i);
  * one GPU - then draws exactly what a plan over the whole vector draws there, and since
  * every bucket has its own norm, the shard's codes and scales are the corresponding
  * slices of the whole vector's. Default 0. first_block >= 0, first_block + ceil(d/512)
- * <= 2^26. Takes effect from the next agc_encode_quantize.
+ * <= 2^26, and a multiple of bucket / 512 for buckets of 1024 and above (a range starts at
+ * a bucket). Takes effect from the next agc_encode_quantize.
  */
 int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block);
 /* 1 if the plan encodes with the TMA-staged kernel, 0 if with the direct-load kernel. */

@@ -114,7 +114,7 @@ __device__ __forceinline__ void add_worker(const AgcDecParams &P, int worker, fl
     float cstep_row[4];
 #pragma unroll
     for (int bk = 0; bk < 4 / RB; ++bk) {
-        const long long beta = P.global_norm ? 0 : q * (4 / RB) + bk;
+        const long long beta = (q * (4 / RB) + bk) >> P.scale_shift;
         const float S = beta < P.nb ? __ldg(P.scales + (long long)worker * P.nb + beta) : 0.0f;
         const float cs = __fmul_rn(__fmul_rn(wgt, S), dstep);
 #pragma unroll
@@ -560,7 +560,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                     const float *srow = P.scales + s_wk[r0 + lane].scales_off;
 #pragma unroll
                     for (int bk = 0; bk < 4 / RB; ++bk) {
-                        const long long beta_idx = P.global_norm ? 0 : q * (4 / RB) + bk;
+                        const long long beta_idx = (q * (4 / RB) + bk) >> P.scale_shift;
                         if (beta_idx < P.nb) sc[bk] = __ldg(srow + beta_idx);
                     }
                 }
@@ -765,7 +765,7 @@ __global__ void __launch_bounds__(512, 1) agc_decode_multi_kernel(const AgcDecPa
         for (int t = 0; t < 4; ++t) pw[t] = t < cnt ? __ldg(src + t) : 0u;
 #pragma unroll
         for (int bk = 0; bk < 4 / RB; ++bk) {
-            const long long beta_idx = P.global_norm ? 0 : q * (4 / RB) + bk;
+            const long long beta_idx = (q * (4 / RB) + bk) >> P.scale_shift;
             ps[bk] = beta_idx < P.nb ? __ldg(P.scales + (long long)e.worker * P.nb + beta_idx) : 0.0f;
         }
     };
@@ -997,7 +997,7 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     P.n = plan->n;
     P.R = R;
     P.rows_per_bucket = plan->bucket / 128;
-    P.global_norm = plan->global_norm ? 1 : 0;
+    P.scale_shift = plan->scale_shift;
     P.lr0 = (beta && lr_host) ? lr_host[0] : 0.0f;
     P.lr = plan->d_lr;
     P.status = status;
@@ -1069,7 +1069,7 @@ int agc_launch_decode_residuals(agc_plan *plan, const void *codes, const float *
     P.n = plan->n;
     P.R = R;
     P.rows_per_bucket = plan->bucket / 128;
-    P.global_norm = plan->global_norm ? 1 : 0;
+    P.scale_shift = plan->scale_shift;
     P.lr0 = 0.0f;
     P.lr = nullptr;
     P.gref = g_ref;
@@ -1126,7 +1126,7 @@ int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *
     P.n = plan->n;
     P.R = 1;
     P.rows_per_bucket = plan->bucket / 128;
-    P.global_norm = plan->global_norm ? 1 : 0;
+    P.scale_shift = plan->scale_shift;
     P.lr0 = 0.0f;
     P.lr = nullptr;
     P.status = status;

@@ -74,7 +74,8 @@ struct AgcEncParams {
     const float *G;
     const float *const *G_rows;  // k row pointers instead of G (direct kernel only), or NULL
     float *partials;             // global norm: n x nblk block sums of squares
-    const float *ginv;           // global norm: n reciprocal scales (0 = flushed worker)
+    const float *ginv;           // two-pass modes: n x nb reciprocal scales (0 = flushed), nb = 1 for the global norm
+    int group_shift = -1;        // buckets of 2^group_shift pack blocks (second pass reads ginv per task), or -1
     uint32_t *codes;
     float *scales;
     uint32_t *status;
@@ -99,7 +100,8 @@ struct AgcDecParams {
     long long d, nblk, nb;
     int n, R;
     int rows_per_bucket;
-    int global_norm = 0;    // one scale per worker: scales[i]
+    int scale_shift = 0;    // scale index of 512-bucket beta = beta >> scale_shift (buckets of 1024+ coordinates: log2 of
+                            // their blocks; one global norm per worker: large enough to give 0)
     float lr0;              // learning rate of the single realisation (R == 1)
     const float *lr;        // device, R learning rates (per-realisation mode with beta)
     uint32_t *status = nullptr;  // AGC_STATUS_* bits are OR-ed into it (ring kernel), may be NULL
@@ -123,6 +125,8 @@ struct agc_plan {
     uint64_t seed = 0;
     long long first_block = 0;
     bool global_norm = false;     // one l2 norm per worker (bucket argument 0)
+    int group_blocks = 0;         // pack blocks per bucket for bucket arguments 1024, 2048, 4096 (else 0)
+    int scale_shift = 0;          // see AgcDecParams
     float *d_partials = nullptr, *d_chunk_sums = nullptr, *d_ginv = nullptr;
     uint32_t flags = 0;
     int device = 0, sm_count = 0;

@@ -128,7 +128,8 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     *out = nullptr;
     if (n_workers < 1 || k_parts < 1 || d < 1 || d > (int64_t(1) << 31) - 1024) return AGC_ERR_ARG;
     if (!row_ptr || !col_idx || !a || !w || !p || !bits) return AGC_ERR_ARG;
-    if (bucket != 0 && bucket != 128 && bucket != 256 && bucket != 512) return AGC_ERR_ARG;
+    if (bucket != 0 && bucket != 128 && bucket != 256 && bucket != 512 && bucket != 1024 && bucket != 2048 && bucket != 4096)
+        return AGC_ERR_ARG;
     if (row_ptr[0] != 0) return AGC_ERR_ARG;
     for (int i = 0; i < n_workers; ++i) {
         if (row_ptr[i + 1] < row_ptr[i]) return AGC_ERR_ARG;
@@ -159,7 +160,10 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     pl->k = k_parts;
     pl->d = d;
     pl->global_norm = bucket == 0;
-    pl->bucket = bucket ? int(bucket) : AGC_BLOCK;   // the global norm runs the 512-block kernels
+    pl->group_blocks = bucket > AGC_BLOCK ? int(bucket / AGC_BLOCK) : 0;
+    // the global norm and the buckets of several pack blocks run the 512-block kernels in two passes
+    pl->bucket = (bucket && bucket <= AGC_BLOCK) ? int(bucket) : AGC_BLOCK;
+    pl->scale_shift = pl->global_norm ? 62 : pl->group_blocks == 8 ? 3 : pl->group_blocks == 4 ? 2 : pl->group_blocks == 2 ? 1 : 0;
     pl->seed = seed;
     pl->flags = flags;
     pl->nblk = (d + AGC_BLOCK - 1) / AGC_BLOCK;
@@ -238,11 +242,11 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     if (!rc) rc = upload(&pl->d_grp_wk_ptr, grp_wk_ptr);
     if (!rc) rc = upload(&pl->d_grp_workers, grp_workers);
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_weff), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
-    if (!rc && pl->global_norm) {
+    if (!rc && (pl->global_norm || pl->group_blocks)) {
         const size_t nchunk = size_t((pl->nblk + 1023) / 1024);
         if (cudaMalloc(reinterpret_cast<void **>(&pl->d_partials), sizeof(float) * size_t(n_workers) * size_t(pl->nblk)) != cudaSuccess ||
             cudaMalloc(reinterpret_cast<void **>(&pl->d_chunk_sums), sizeof(float) * size_t(n_workers) * nchunk) != cudaSuccess ||
-            cudaMalloc(reinterpret_cast<void **>(&pl->d_ginv), sizeof(float) * n_workers) != cudaSuccess)
+            cudaMalloc(reinterpret_cast<void **>(&pl->d_ginv), sizeof(float) * size_t(n_workers) * size_t(pl->nb)) != cudaSuccess)
             rc = AGC_ERR_NOMEM;
     }
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_v), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
@@ -275,6 +279,7 @@ extern "C" size_t agc_worker_offset(const agc_plan_t *plan, int i)
 extern "C" int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block)
 {
     if (!plan || first_block < 0 || first_block + plan->nblk > (int64_t(1) << 26)) return AGC_ERR_ARG;
+    if (plan->group_blocks && first_block % plan->group_blocks) return AGC_ERR_ARG;   // a range starts at a bucket
     plan->first_block = first_block;
     return AGC_OK;
 }

@@ -633,6 +633,73 @@ def test_residuals_of_many_realisations_without_storing_g_hat(agc, torch, R, B, 
     assert (np.abs(got - want) <= 1e-6 * want).all()
 
 
+@pytest.mark.parametrize("B,d,direct", [(1024, 300, False), (1024, 70_001, False), (2048, 5000, True), (2048, 600_001, False),
+                                        (4096, 40_000, False), (4096, 4096 * 3 + 1, True)])
+def test_buckets_of_several_pack_blocks(agc, torch, B, d, direct):
+    """Buckets of 1024, 2048 and 4096 coordinates (2, 4, 8 pack blocks; two passes like the global
+    norm): messages and scales against the oracle's grouped encoder bit for bit, then every
+    decoder on them: single realisation with the fused update, nine realisations in one pass,
+    the collapsed update and the two-track decode."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(B + d)
+    n = k = 7
+    bits = np.array([1, 2, 3, 4, 5, 6, 8], np.uint8)
+    p = rng.uniform(0.05, 0.4, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, 512)
+    G_host = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 2, (k, 1))).astype(np.float32)
+    if d > 3 * B:
+        G_host[:, B:2 * B] = 0.0                       # a bucket that every worker sends as zeros
+    flags = agc.AGC_FLAG_ALLOW_1BIT | (agc.AGC_FLAG_FORCE_DIRECT if direct else 0)
+    ses = Session(n, k, d, rp, ci, a, w, p, bits, bucket=B, seed=17, flags=flags)
+    ld = (d + 3) // 4 * 4
+    G = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+    G[:, :d] = torch.from_numpy(G_host)
+    ses.codes.fill_(-1)
+    ses.scales.fill_(-1.0)
+    for rnd in (0, 4):
+        ses.encode(G, rnd)
+    torch.cuda.synchronize()
+    assert int(ses.status.item()) == 0 and ses.uses_tma == (not direct)
+    oc, osc, st, _ = orp.encode_quantize_grouped(rp, ci, a, bits, B, 17, 4, G_host)
+    assert st == 0
+    assert ses.scales_host().shape == osc.shape
+    assert (ses.scales_host().view(np.uint32) == osc.view(np.uint32)).all()
+    bad = np.nonzero(ses.codes_host() != oc)[0]
+    assert bad.size == 0, f"{bad.size} code words differ, first at {bad[:5]}"
+    if d > 3 * B:
+        assert (osc[:, 1] == 0.0).all()
+    per_block = orp.expand_grouped_scales(osc, d, B)
+    R = 9
+    masks = (rng.random((R, n)) >= p).astype(np.uint8)
+    lr = rng.uniform(1e-3, 1e-1, R).astype(np.float32)
+    beta0 = rng.standard_normal(d).astype(np.float32)
+    og, ob = orp.decode(d, bits, 512, w, masks, oc, per_block, lr=lr, beta=beta0)
+    m_dev = torch.from_numpy(masks).cuda()
+    ghat = torch.full((R, d), -3.0, dtype=torch.float32, device="cuda")
+    ses.decode(m_dev, ghat=ghat)                                     # nine realisations in one pass
+    assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
+    g1 = torch.empty((1, d), dtype=torch.float32, device="cuda")
+    b1 = torch.from_numpy(beta0.copy()).cuda()
+    ses.decode(m_dev[:1], lr=lr[:1], ghat=g1, beta=b1)                # one realisation, fused update
+    og1, ob1 = orp.decode(d, bits, 512, w, masks[:1], oc, per_block, lr=lr[:1], beta=beta0)
+    assert (g1.cpu().numpy().view(np.uint32) == og1.view(np.uint32)).all()
+    assert (b1.cpu().numpy().view(np.uint32) == ob1.view(np.uint32)).all()
+    b2 = torch.from_numpy(beta0.copy()).cuda()
+    ses.decode(m_dev, lr=lr, beta=b2)                                # collapsed update
+    assert np.abs(b2.cpu().numpy() - ob).max() / np.abs(ob).max() <= 1e-5
+    if not direct:
+        v2 = (0.5 * w).astype(np.float32)
+        gw = torch.empty(d, dtype=torch.float32, device="cuda")
+        gv = torch.empty(d, dtype=torch.float32, device="cuda")
+        agc.agc_decode_two_track(ses.plan, ses.codes, ses.scales, m_dev[0], v2, gw, gv, status_dev=ses.status)
+        ogv, _ = orp.decode(d, bits, 512, v2, masks[:1], oc, per_block)
+        assert (gw.cpu().numpy().view(np.uint32) == og[0].view(np.uint32)).all()
+        assert (gv.cpu().numpy().view(np.uint32) == ogv[0].view(np.uint32)).all()
+    torch.cuda.synchronize()
+    assert int(ses.status.item()) == 0
+    ses.close()
+
+
 @pytest.mark.parametrize("kind", ["cyclic", "interval"])
 def test_lemma1_bound_and_unbiasedness_measured_on_the_gpu(agc, torch, kind):
     """Lemma 1 as a measured experiment: 20 rounds x 64 straggler realisations through the CUDA
