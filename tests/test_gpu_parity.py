@@ -697,6 +697,10 @@ def test_buckets_of_several_pack_blocks(agc, torch, B, d, direct):
         assert (gv.cpu().numpy().view(np.uint32) == ogv[0].view(np.uint32)).all()
     torch.cuda.synchronize()
     assert int(ses.status.item()) == 0
+    with pytest.raises(agc.AgcError) as e:       # a range of a longer vector starts at a bucket
+        ses.set_first_block(B // 512 + 1)
+    assert e.value.code == -1
+    ses.set_first_block(3 * (B // 512))
     ses.close()
 
 
