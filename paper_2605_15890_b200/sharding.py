@@ -9,7 +9,8 @@ BLOCK = 512
 
 def coordinate_range(d_total, rank, world, align=BLOCK):
     """[start, stop) of rank's shard: whole pack blocks, as equal as possible, the last
-    shard taking the ragged tail. Shards of ranks 0..world-1 tile [0, d_total)."""
+    shard taking the ragged tail. Shards of ranks 0..world-1 tile [0, d_total). With buckets of
+    more than 512 coordinates pass the bucket size as `align`: a shard starts at a bucket."""
     if not (0 <= rank < world) or d_total < 0:
         raise ValueError("bad rank / size")
     nblk = (d_total + align - 1) // align
@@ -21,7 +22,7 @@ def coordinate_range(d_total, rank, world, align=BLOCK):
 
 def first_block(d_total, rank, world, align=BLOCK):
     """Pack-block index of the shard's first coordinate (for agc_plan_set_first_block)."""
-    return coordinate_range(d_total, rank, world, align)[0] // align
+    return coordinate_range(d_total, rank, world, align)[0] // BLOCK
 
 
 def max_over_ranks(values, device=None):

@@ -100,3 +100,19 @@ def test_coordinate_ranges_tile_the_vector(d, world):
     sizes = [sharding.coordinate_range(d, r, world) for r in range(world)]
     blocks = [(hi - lo + 511) // 512 for lo, hi in sizes]
     assert max(blocks) - min(blocks) <= 1
+
+
+@pytest.mark.parametrize("d,world,B", [(25_557_032, 8, 1024), (10**7 + 3, 3, 4096), (5000, 4, 2048)])
+def test_ranges_aligned_to_buckets_of_several_blocks(d, world, B):
+    """With buckets above 512 coordinates a shard starts at a bucket and first_block still counts
+    pack blocks (a multiple of the blocks per bucket, which agc_plan_set_first_block requires)."""
+    prev = 0
+    for r in range(world):
+        lo, hi = sharding.coordinate_range(d, r, world, align=B)
+        assert lo == prev and lo <= hi <= d
+        assert lo % B == 0 or lo == d
+        fb = sharding.first_block(d, r, world, align=B)
+        assert fb * 512 == lo or lo == d
+        assert fb % (B // 512) == 0 or lo == d
+        prev = hi
+    assert prev == d
