@@ -312,7 +312,9 @@ def main():
     # weak scaling: the job is a gradient of world * nblk pack blocks, rank r holds blocks
     # [r * nblk, (r + 1) * nblk) of it (its own data, same shape), no exchange on the data path
     ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, bits, bucket=bucket, seed=wl.seed, flags=flags, device=dev)
-    ses.set_first_block(sharding.first_block(world * ((wl.d + 511) // 512) * 512, rank, world))
+    align = max(512, bucket)                                  # a rank's range starts at a bucket
+    per_rank = (wl.d + align - 1) // align * align
+    ses.set_first_block(sharding.first_block(world * per_rank, rank, world, align=align))
     wl.seed += 7919 * rank  # the synthetic values of this rank's range
     ld = (wl.d + 3) // 4 * 4
     G = cfgs.partials_torch(wl, dev, ld=ld)
