@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
 same seeded inputs. Packed codes, scales and the single-realisation decode must be
 bit-exact; the collapsed multi-realisation update must agree to 1e-5 relative."""
+import os
+
 import numpy as np
 import pytest
 
@@ -59,8 +61,17 @@ def run_both(agc, torch, G_host, code, p, bits, B, seed, rnd, masks, flags=0, d=
         out["beta_fused"] = b2.cpu().numpy()
     torch.cuda.synchronize()
     ses.close()
-    oc, osc, ost, _ = orp.encode_quantize(rp, ci, a, bits, B, seed, rnd, G_host[:, :d], d=d)
-    og, ob = orp.decode(d, bits, B, w, masks, oc, osc, lr=lr, beta=beta0)
+    Gd = np.ascontiguousarray(G_host[:, :d])
+    if B == 0:        # one norm per worker
+        oc, osc, ost, _ = orp.encode_quantize_global(rp, ci, a, bits, seed, rnd, Gd, d=d)
+        dec_scales, dec_B, osc = orp.expand_global_scales(osc, d), 512, osc.reshape(n, 1)
+    elif B > 512:     # buckets of several pack blocks
+        oc, osc, ost, _ = orp.encode_quantize_grouped(rp, ci, a, bits, B, seed, rnd, Gd, d=d)
+        dec_scales, dec_B = orp.expand_grouped_scales(osc, d, B), 512
+    else:
+        oc, osc, ost, _ = orp.encode_quantize(rp, ci, a, bits, B, seed, rnd, Gd, d=d)
+        dec_scales, dec_B = osc, B
+    og, ob = orp.decode(d, bits, dec_B, w, masks, oc, dec_scales, lr=lr, beta=beta0)
     ref = dict(codes=oc, scales=osc, ghat=og, status=ost, beta=ob)
     return out, ref
 
@@ -171,7 +182,7 @@ def test_code_structures(agc, torch, kind):
     assert G.shape[0] == k
 
 
-@pytest.mark.parametrize("case", range(16))
+@pytest.mark.parametrize("case", range(int(os.environ.get("AGC_SWEEP_CASES", "16"))))   # more cases for a longer sweep
 def test_seeded_random_shapes_codes_and_masks(agc, torch, case):
     """Random worker / partition counts, sparse supports, widths, bucket sizes, lengths (a few
     blocks up to several hundred: every tile height of the decoder), heavy-tailed values, 64-bit
@@ -179,7 +190,7 @@ def test_seeded_random_shapes_codes_and_masks(agc, torch, case):
     rng = np.random.default_rng(9000 + case)
     n = int(rng.integers(1, 70))
     k = int(rng.integers(1, 50))
-    B = int(rng.choice([128, 256, 512]))
+    B = int(rng.choice([128, 256, 512, 512, 1024, 2048, 4096, 0]))
     d = int(rng.choice([rng.integers(1, 3000), rng.integers(3000, 80_000), rng.integers(80_000, 400_000)]))
     if n * d > 6_000_000:
         d = 6_000_000 // n
