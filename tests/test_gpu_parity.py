@@ -209,6 +209,8 @@ def test_seeded_random_shapes_codes_and_masks(agc, torch, case):
     if case % 4 == 0:
         G[rng.integers(0, k), : min(d, 600)] = 0.0          # stretches of zeros inside a row
     R = int(rng.integers(1, 5))
+    if case % 3 == 0 and n * d <= 400_000:
+        R = int(rng.integers(8, 70))                        # g_hat of all realisations in one pass
     masks = (rng.random((R, n)) >= p).astype(np.uint8)
     lr = rng.uniform(1e-3, 1e-1, R).astype(np.float32)
     beta0 = rng.standard_normal(d).astype(np.float32)
