@@ -491,7 +491,9 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     }
     __syncthreads();
     const int n_groups = flags[2];
-    const long long ntile = (P.nblk + qt - 1) / qt;
+    // block and tile indices fit 32 bits (d < 2^31 coordinates)
+    const int nblk = (int)P.nblk;
+    const int ntile = (int)((P.nblk + qt - 1) / qt);
 
     if (warp == QT) {
         // ---------------- producer
@@ -499,9 +501,9 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         int s = 0;
         uint32_t parity = 1;
         bool ok = true;
-        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q0 = T * qt;
-            const uint32_t nq = (uint32_t)(P.nblk - q0 < qt ? P.nblk - q0 : qt);
+        for (int T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+            const int q0 = T * (int)qt;
+            const uint32_t nq = (uint32_t)(nblk - q0) < qt ? (uint32_t)(nblk - q0) : qt;
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 uint32_t bytes = 0, soff = 0, wbits = 0;
@@ -511,7 +513,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                     wbits = wk.bits;
                     bytes = nq * 64u * wk.bits;
                     soff = wk.soff;
-                    src = reinterpret_cast<const unsigned char *>(P.codes + wk.word_off + q0 * 16 * wk.bits);
+                    src = reinterpret_cast<const unsigned char *>(P.codes + wk.word_off + (long long)(q0 * 16 * (int)wk.bits));
                 }
                 uint32_t total = bytes;
 #pragma unroll
@@ -526,8 +528,8 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                     // the same workers' chunks of this CTA's next tile row: on their way to L2 a
                     // whole tile row ahead, so that the ring refills at L2 latency, not HBM latency
                     const long long qn = q0 + (long long)gridDim.x * qt;
-                    if (qn < P.nblk) {
-                        const uint32_t nqn = (uint32_t)(P.nblk - qn < qt ? P.nblk - qn : qt);
+                    if (qn < nblk) {
+                        const uint32_t nqn = (uint32_t)(nblk - qn) < qt ? (uint32_t)(nblk - qn) : qt;
                         bulk_prefetch_l2(src + (size_t)gridDim.x * qt * 64u * wbits, nqn * 64u * wbits);
                     }
 #endif
@@ -550,17 +552,17 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         bool ok = true;
         // scales of the lane's worker (lane < workers of the group) for this warp's block of a
         // tile; fetched one tile ahead so that their latency hides behind the current tile
-        auto fetch_scales = [&](long long T, int g, float (&sc)[4 / RB]) {
+        auto fetch_scales = [&](int T, int g, float (&sc)[4 / RB]) {   // T may lie one step past the last tile
 #pragma unroll
             for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
-            const long long q = T * qt + warp;
-            if (T < ntile && g < n_groups && (uint32_t)warp < qt && q < P.nblk) {
+            const int q = T * (int)qt + warp;
+            if (T < ntile && g < n_groups && (uint32_t)warp < qt && q < nblk) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
                 if (lane < nr) {
                     const float *srow = P.scales + s_wk[r0 + lane].scales_off;
 #pragma unroll
                     for (int bk = 0; bk < 4 / RB; ++bk) {
-                        const long long beta_idx = (q * (4 / RB) + bk) >> P.scale_shift;
+                        const int beta_idx = (q * (4 / RB) + bk) >> P.scale_shift;   // < 2^24
                         if (beta_idx < P.nb) sc[bk] = __ldg(srow + beta_idx);
                     }
                 }
@@ -568,9 +570,9 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         };
         float sc_next[4 / RB];
         fetch_scales(blockIdx.x, 0, sc_next);
-        for (long long T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
-            const long long q = T * qt + warp;
-            const bool active = (uint32_t)warp < qt && q < P.nblk;
+        for (int T = blockIdx.x; ok && T < ntile; T += gridDim.x) {
+            const int q = T * (int)qt + warp;
+            const bool active = (uint32_t)warp < qt && q < nblk;
             float acc[16], acc2[16], b[16];   // acc2: second track, unused and dropped in the other modes
 #pragma unroll
             for (int t = 0; t < 16; ++t) acc[t] = 0.0f;
