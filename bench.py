@@ -112,7 +112,7 @@ class ClockSampler:
         except Exception:
             pass
         self.th.join(timeout=5)
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         for ln in self.lines:
             f = [t.strip() for t in ln.split(",")]
             if len(f) < 9:
@@ -121,11 +121,15 @@ class ClockSampler:
                 sm.append(float(f[1])); smax.append(float(f[2]))
             except ValueError:
                 continue
+            try:
+                power.append(float(f[3]))
+            except ValueError:
+                pass
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "power_w_max": max(power) if power else None}
 
 
 def oracle_round(orp, code, bits, bucket, seed, t, G, d, mask, lr, beta):
