@@ -16,7 +16,7 @@
  * Notation: n workers, k partitions, d coordinates, b_i bits of worker i,
  * L_i = 2^(b_i-1) - 1 magnitude levels (the paper's s_i), B bucket size.
  *
- * Wire format (the paper only counts bits; the layout is this build's):
+ * Wire format (the paper only counts bits; the layout is this library's):
  *   - coordinates are grouped in pack blocks of 512; inside a block the
  *     coordinate with offset o = 128*c + 4*l + e (c<4, l<32, e<4) sits at
  *     stream position 16*l + 4*c + e;

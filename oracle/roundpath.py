@@ -1,7 +1,7 @@
 """numpy front end of the C oracle for the per-round path (test infrastructure).
 
 Argument marshalling only; all arithmetic is in agc_oracle.c. Notation follows
-the paper's Sec. II with this build's letters: n workers, k partitions,
+the paper's Sec. II with these letters: n workers, k partitions,
 d coordinates, bits b_i, bucket size B.
 """
 import ctypes as C
