@@ -226,15 +226,34 @@ def build_code(agc, wl, bucket):
     return (rp, ci, a, w), np.asarray(bits, np.uint8)
 
 
+def oracle_build_code(wl, bucket):
+    """Bits and code weights of the workload from the oracle's own design code (float64 numpy /
+    scipy): Algorithm 1 for the bits, the support-restricted problem (c-SP2) for the weights.
+    Used by the reference arm, which must not touch the CUDA library."""
+    from oracle import design as od
+    phi_dim = float(bucket) if bucket else 512.0
+    if wl.bits is None:
+        bits, _ = od.bit_allocate_low_complexity(wl.p, wl.z_tot, phi_dim, b_max=wl.bits_range[1])
+    else:
+        bits = wl.bits
+    bits = np.asarray(bits, np.uint8)
+    support = od.cyclic_support(wl.n, wl.k, wl.s)
+    c = od.c_coeff(wl.p, bits, phi_dim)
+    alpha, _ = od.support_restricted_alpha_reference(c, support, wl.k)
+    rp, ci, vals = od.alpha_to_csr(alpha, drop=1e-9)
+    _, w = od.physical_coefficients(alpha, wl.p)
+    return (rp, ci, vals.astype(np.float32), w.astype(np.float32)), bits
+
+
 def run_reference(args, wl, bucket):
-    """Reference arm: the CPU oracle as it stands, on host cores, each step a bounded sample."""
+    """Reference arm: the CPU oracle as it stands, on host cores, each step a bounded sample.
+    Nothing of the CUDA library is imported here: bits and weights come from oracle/design.py."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import paper_2605_15890_b200 as agc  # host-only design calls (no GPU work)
     from oracle import roundpath as orp
     from synth import configs as cfgs
-    code, bits = build_code(agc, wl, bucket)
+    code, bits = oracle_build_code(wl, bucket)
     rp, ci, a, w = code
     rate0, _, _ = oracle_sample_rate(wl, code, bits, bucket, target_s=2.0)
     # the whole run (warm-up + timed steps) is sized to about two minutes of host time

@@ -94,22 +94,30 @@ static float dec_offset(int b) { return b >= 2 ? (float)((1 << (b - 1)) - 1) : 0
 static float dec_step(int b)   { return b >= 2 ? (float)(1.0 / (double)((1 << (b - 1)) - 1)) : 2.0f; }
 static uint32_t zero_code(int b) { return b >= 2 ? (uint32_t)((1 << (b - 1)) - 1) : 0u; }
 
-static inline uint32_t f2u(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
-
-/* Eq. rv_quant for one coordinate. inv = enc_scale(b)/S. With y = L*x/S the
- * paper's rule (level floor(y) or floor(y)+1, the latter w.p. y - floor(y))
- * is level = floor(y + r) for r uniform in [0,1); it also holds for negative y,
- * so the sign needs no separate treatment. r = u/2^15, and the sum is formed
- * in fixed point with 15 fractional bits inside the mantissa of a float in
- * [2^23, 2^24): one correctly rounded fma gives round(x*inv) + offset + u.
- * Returns the offset-binary code level + L (b >= 2), or the bit of the
- * two-point quantiser (b == 1), before masking to b bits. */
+/* Eq. rv_quant for one coordinate, written out. inv = enc_scale(b)/S, so
+ * y = x*inv is L*x/S counted in units of 2^-15 of a level step. The paper's rule
+ * (level floor(y) or floor(y)+1, the latter w.p. y - floor(y)) is
+ * level = floor(y + r) for r uniform in [0,1); it also holds for negative y, so
+ * the sign needs no separate treatment. Here r = u/2^15 with a 15-bit integer u,
+ * and y is kept to 15 fractional bits:
+ *     t     = y + offset + u           (offset = L*2^15 makes every code >= 0)
+ *     fixed = t rounded to the nearest integer, ties to the even integer
+ *     code  = floor(fixed / 2^15)      = level + L
+ * Everything below is exact: the product of two floats is a double (24 x 24
+ * significant bits), floor(y) and the integer part of t are exact, and the
+ * fractional part of y decides the rounding by comparison with 1/2.
+ * Returns the offset-binary code level + L (b >= 2), or the bit of the two-point
+ * quantiser (b == 1: offset = 2^14, inv = 2^14/S, so t/2^15 = (1 + x/S)/2 + r),
+ * before masking to b bits. */
 uint32_t agc_oracle_quantize_one(float x, float inv, int b, uint32_t u)
 {
-    float addend = (float)(8388608u + enc_offset(b) + u); /* exact: an integer below 2^24 */
-    float tq = fmaf(x, inv, addend);
-    uint32_t fixed = f2u(tq) - 0x4B000000u;
-    return fixed >> AGC_FRAC_BITS;
+    double y = (double)x * (double)inv;
+    double fl = floor(y);
+    double frac = y - fl;                                /* in [0, 1] */
+    int64_t whole = (int64_t)fl + (int64_t)enc_offset(b) + (int64_t)u;   /* integer part of t */
+    int up = frac > 0.5 || (frac == 0.5 && (whole & 1)); /* nearest, ties to even */
+    int64_t fixed = whole + up;
+    return (uint32_t)(fixed >> AGC_FRAC_BITS);           /* fixed >= 0: the shift is the floor */
 }
 
 /* the fp32 reciprocal scale the encoder multiplies by: enc_scale(b) / S */

@@ -562,7 +562,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                     const float *srow = P.scales + s_wk[r0 + lane].scales_off;
 #pragma unroll
                     for (int bk = 0; bk < 4 / RB; ++bk) {
-                        const int beta_idx = (q * (4 / RB) + bk) >> P.scale_shift;   // < 2^24
+                        const long long beta_idx = ((long long)q * (4 / RB) + bk) >> P.scale_shift;
                         if (beta_idx < P.nb) sc[bk] = __ldg(srow + beta_idx);
                     }
                 }
@@ -1090,8 +1090,9 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
     plan->dec_stages = ring_layout<AGC_DEC_QT>(plan->n, smem_optin, &plan->dec_smem, &plan->dec_w2_offset);
     plan->dec2_stages = ring_layout<AGC_DEC_QT2>(plan->n, smem_optin, &plan->dec2_smem, &plan->dec2_w2_offset);
     if (plan->dec_stages < 2 || plan->dec2_stages < 2) return AGC_OK;
-    if (!ring_set_smem<0, AGC_DEC_QT>(int(plan->dec_smem)) || !ring_set_smem<1, AGC_DEC_QT>(int(plan->dec_smem)) ||
-        !ring_set_smem<2, AGC_DEC_QT2>(int(plan->dec2_smem)))
+    // the limit is an attribute of the kernel, shared by all plans: the device's opt-in maximum
+    if (!ring_set_smem<0, AGC_DEC_QT>(smem_optin) || !ring_set_smem<1, AGC_DEC_QT>(smem_optin) ||
+        !ring_set_smem<2, AGC_DEC_QT2>(smem_optin))
         return AGC_ERR_CUDA;
     if (cudaFuncSetAttribute(agc_decode_multi_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
         cudaFuncSetAttribute(agc_decode_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||

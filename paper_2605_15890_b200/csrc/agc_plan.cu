@@ -6,7 +6,7 @@
 
 #include "agc_internal.h"
 
-int agc_encode_prepare(agc_plan *plan);
+int agc_encode_prepare(agc_plan *plan, int smem_optin);
 int agc_decode_prepare(agc_plan *plan, int smem_optin);
 
 namespace {
@@ -251,7 +251,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     }
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_v), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_lr), sizeof(float) * AGC_MAX_R) != cudaSuccess) rc = AGC_ERR_NOMEM;
-    if (!rc) rc = agc_encode_prepare(pl);
+    if (!rc) rc = agc_encode_prepare(pl, smem_optin);
     if (!rc) rc = agc_decode_prepare(pl, smem_optin);
     if (rc) {
         free_device(pl);
@@ -280,6 +280,9 @@ extern "C" int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block)
 {
     if (!plan || first_block < 0 || first_block + plan->nblk > (int64_t(1) << 26)) return AGC_ERR_ARG;
     if (plan->group_blocks && first_block % plan->group_blocks) return AGC_ERR_ARG;   // a range starts at a bucket
+    // one norm per worker over the WHOLE vector (Eq. quant_def): a range of it cannot be
+    // encoded on its own, its norm would be the range's
+    if (plan->global_norm && first_block != 0) return AGC_ERR_STATE;
     plan->first_block = first_block;
     return AGC_OK;
 }
@@ -367,7 +370,15 @@ extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_
                   cudaMalloc(reinterpret_cast<void **>(&plan->h_ghat), sizeof(float) * plan->d) == cudaSuccess &&
                   cudaMalloc(reinterpret_cast<void **>(&plan->h_mask), plan->n) == cudaSuccess &&
                   cudaMalloc(reinterpret_cast<void **>(&plan->h_status), sizeof(uint32_t)) == cudaSuccess;
-        if (!ok) return AGC_ERR_NOMEM;
+        if (!ok) {
+            // leave no half-allocated staging behind: the next call starts over
+            cudaFree(plan->h_G); cudaFree(plan->h_codes); cudaFree(plan->h_scales);
+            cudaFree(plan->h_ghat); cudaFree(plan->h_mask); cudaFree(plan->h_status);
+            plan->h_G = nullptr; plan->h_codes = nullptr; plan->h_scales = nullptr;
+            plan->h_ghat = nullptr; plan->h_mask = nullptr; plan->h_status = nullptr;
+            cudaGetLastError();
+            return AGC_ERR_NOMEM;
+        }
     }
     if (cudaMemcpy2DAsync(plan->h_G, sizeof(float) * ld_dev, G_host, sizeof(float) * ld_host,
                           sizeof(float) * plan->d, plan->k, cudaMemcpyHostToDevice, st) != cudaSuccess ||
