@@ -15,7 +15,7 @@ _BINDING_NAMES = (
     "agc_bit_allocate", "agc_bit_allocate_dp", "agc_code_build", "agc_codes_bytes", "agc_decode",
     "agc_decode_two_track", "agc_decode_update_static", "agc_decode_residuals", "agc_two_track_vector", "AGC_ERR_LIMIT",
     "agc_encode_quantize", "agc_encode_quantize_rows", "agc_eta_balance", "agc_plan_create", "agc_plan_destroy", "agc_plan_set_first_block", "agc_plan_uses_tma",
-    "agc_round_host", "agc_scales_bytes", "agc_selftest_division", "agc_strerror", "agc_version", "agc_worker_offset",
+    "agc_round_host", "agc_scales_bytes", "agc_selftest_division", "agc_selftest_sqrt", "agc_strerror", "agc_version", "agc_worker_offset",
     "library_path")
 
 __all__ = list(_BINDING_NAMES)

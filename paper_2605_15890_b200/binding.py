@@ -87,6 +87,8 @@ def _load():
     L.agc_code_build.restype = C.c_int
     L.agc_selftest_division.argtypes = [C.POINTER(C.c_ulonglong)]
     L.agc_selftest_division.restype = C.c_int
+    L.agc_selftest_sqrt.argtypes = [C.POINTER(C.c_ulonglong)]
+    L.agc_selftest_sqrt.restype = C.c_int
     L.agc_eta_balance.argtypes = [C.c_int, f64p, C.c_int, C.c_double, f64p]
     L.agc_eta_balance.restype = C.c_int
     L.agc_strerror.argtypes = [C.c_int]
@@ -260,6 +262,14 @@ def agc_selftest_division():
     correctly rounded quotient (expected 0)."""
     bad = C.c_ulonglong(0)
     _check(_lib.agc_selftest_division(C.byref(bad)))
+    return bad.value
+
+
+def agc_selftest_sqrt():
+    """Number of normal floats whose square root in the encoder differs from the correctly
+    rounded one (expected 0)."""
+    bad = C.c_ulonglong(0)
+    _check(_lib.agc_selftest_sqrt(C.byref(bad)))
     return bad.value
 
 

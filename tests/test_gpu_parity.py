@@ -268,6 +268,34 @@ def test_nonfinite_and_zero_buckets(agc, torch):
     assert ((out["ghat"].view(np.uint32) == ref["ghat"].view(np.uint32)) | both_nan).all()
 
 
+@pytest.mark.parametrize("B", [128, 256, 512, 2048, 0])
+@pytest.mark.parametrize("direct", [False, True])
+def test_buckets_with_tiny_sums_of_squares(agc, torch, B, direct):
+    """Sums of squares across the whole exponent range: ordinary, between the smallest normal
+    number and 2^-102 (the encoder's general square root and division), below the smallest normal
+    (flushed), huge. Blocks differ in magnitude, so every path occurs in one message."""
+    rng = np.random.default_rng(31 + B)
+    n = k = 6
+    d = 16 * 512 + 77
+    bits = np.array([1, 2, 3, 4, 6, 8], np.uint8)
+    p = np.full(n, 0.1)
+    code = _codes.cyclic_code(p, bits, k, 2, 512)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    mags = [1.0, 1e-15, 3e-17, 1e-18, 2e-19, 1e-20, 1e-22, 1e17, 3e-16, 7e-17, 1e-17, 5e-18, 4e-19, 1e-19, 1e5, 1e-25, 1.0]
+    for q, m in enumerate(mags):
+        G[:, q * 512:(q + 1) * 512] *= np.float32(m)
+    G[:, 3 * 512 + 128:3 * 512 + 256] = 0.0      # a flushed 128-bucket next to tiny ones
+    out, ref = run_both(agc, torch, G, code, p, bits, B, 3, 1, np.ones((1, n)),
+                        flags=agc.AGC_FLAG_FORCE_DIRECT if direct else 0)
+    assert out["status"] == 0 and ref["status"] == 0
+    assert (out["scales"].view(np.uint32) == ref["scales"].view(np.uint32)).all()
+    if B in (128, 256, 512):
+        tiny = (ref["scales"] > 0) & (ref["scales"] < 2.0 ** -51)
+        assert tiny.any() and (ref["scales"] == 0).any()
+    assert (out["codes"] == ref["codes"]).all()
+    assert (out["ghat"].view(np.uint32) == ref["ghat"].view(np.uint32)).all()
+
+
 def test_same_round_same_bits_other_round_other_bits(agc, torch):
     wl = cfgs.config1()
     code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
@@ -428,6 +456,12 @@ def test_encoder_division_is_correctly_rounded_everywhere(agc):
     """The encoder's branch-free L 2^15 / S against the IEEE quotient for all eight
     numerators and every float S in [2^-63, 2^64)."""
     assert agc.agc_selftest_division() == 0
+
+
+def test_encoder_square_root_is_correctly_rounded_everywhere(agc):
+    """The encoder's branch-free square root against the IEEE one on its whole domain (every
+    float from 2^-102 up)."""
+    assert agc.agc_selftest_sqrt() == 0
 
 
 def test_config4_least_squares_descent_in_lock_step(agc, torch):
@@ -1035,3 +1069,43 @@ def test_encode_from_separate_row_buffers(agc, torch, B):
     assert bool((ses.codes == want_codes).all()) and bool((ses.scales.view(torch.int32) == want_scales.view(torch.int32)).all())
     assert int(ses.status.item()) == 0
     ses.close()
+
+
+def test_two_live_plans_of_different_shapes_alternate(agc, torch):
+    """Plans of different worker counts and support widths need different amounts of dynamic
+    shared memory from the same kernels; the second plan's creation must not lower the
+    limit the first one launches with. Encode and decode alternate between the two, each
+    checked against the oracle."""
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(77)
+    shapes = [(96, 96, 5, 20_000), (5, 5, 2, 20_000)]       # (n, k, s, d): large tables first, small second
+    plans = []
+    for n, k, s, d in shapes:
+        bits = rng.integers(2, 9, n).astype(np.uint8)
+        p = rng.uniform(0.05, 0.4, n)
+        code = _codes.cyclic_code(p, bits, k, s, 512)
+        G = rng.standard_normal((k, d)).astype(np.float32)
+        mask = (rng.random((1, n)) > 0.2).astype(np.uint8)
+        plans.append(dict(n=n, k=k, d=d, bits=bits, p=p, code=code, G=G, mask=mask))
+    for pl in plans:     # both created before any launch
+        rp, ci, a, w = pl["code"]
+        pl["ses"] = Session(pl["n"], pl["k"], pl["d"], rp, ci, a, w, pl["p"], pl["bits"], bucket=512, seed=9)
+        pl["Gd"] = torch.from_numpy(pl["G"]).cuda()
+        pl["md"] = torch.from_numpy(pl["mask"]).cuda()
+    assert plans[0]["ses"].uses_tma and plans[1]["ses"].uses_tma
+    for rnd in range(3):
+        for pl in plans:
+            ses = pl["ses"]
+            rp, ci, a, w = pl["code"]
+            ghat = torch.empty((1, pl["d"]), dtype=torch.float32, device="cuda")
+            ses.encode(pl["Gd"], rnd)
+            ses.decode(pl["md"], ghat=ghat)
+            torch.cuda.synchronize()
+            oc, osc, _, _ = orp.encode_quantize(rp, ci, a, pl["bits"], 512, 9, rnd, pl["G"])
+            og, _ = orp.decode(pl["d"], pl["bits"], 512, w, pl["mask"], oc, osc)
+            assert int(ses.status.item()) == 0
+            assert (ses.codes_host() == oc).all()
+            assert (ses.scales_host().view(np.uint32) == osc.view(np.uint32)).all()
+            assert (ghat.cpu().numpy().view(np.uint32) == og.view(np.uint32)).all()
+    for pl in plans:
+        pl["ses"].close()
