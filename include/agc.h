@@ -376,11 +376,11 @@ int agc_eta_balance(int n, const double *p, int Z_tot, double phi_dim, double *e
 int agc_selftest_division(unsigned long long *mismatches_out);
 /*
  * agc_selftest_sqrt - diagnostic. The norm of Eq. quant_def is the IEEE-754 correctly rounded
- * square root of the bucket's sum of squares; for sums of at least 2^-102 the encoder
- * computes it with its own branch-free routine (smaller sums take the general one). This
- * call compares the two on the current device for every float of that range (about 1.9e9
- * values) and writes the number of differing results (expected 0) to *mismatches_out (host).
- * Synchronous; allocates 8 bytes of device memory for the duration of the call.
+ * square root of the bucket's sum of squares; the encoder computes it with its own
+ * branch-free routine (sums below 2^-102 are scaled by 2^64 first). This call compares it
+ * on the current device with the IEEE square root for every normal positive float (about
+ * 2.1e9 values) and writes the number of differing results (expected 0) to *mismatches_out
+ * (host). Synchronous; allocates 8 bytes of device memory for the duration of the call.
  */
 int agc_selftest_sqrt(unsigned long long *mismatches_out);
 

@@ -81,7 +81,7 @@ struct AgcEncParams {
     uint32_t *status;
     long long d, ld, nblk, nb;
     long long first_block;       // pack-block index of coordinate 0 in the random stream
-    int n, k, n_groups, nnz;
+    int n, k, n_groups, nnz, n_ops;
     int stages, stage_rows;
     uint32_t round_lo, round_hi;
     uint32_t rk[20];             // Philox round keys: rk[2r] = key0 + r*W0, rk[2r+1] = key1 + r*W1
@@ -136,7 +136,7 @@ struct agc_plan {
     std::vector<long long> word_off;
     // encode tiling
     bool use_tma = false;
-    int n_groups = 0, stage_rows = 0, stages = 0;
+    int n_groups = 0, stage_rows = 0, stages = 0, n_ops = 0;
     size_t enc_smem = 0;
     // decode ring
     bool dec_ring = false;

@@ -208,8 +208,11 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
         edesc[e].a = a[e];
         edesc[e].off = stageable ? uint32_t(ent_slot[e]) * 1024u : 0u;
     }
-    const size_t table_bytes = sizeof(AgcWorkerDesc) * n_workers + sizeof(AgcEntryDesc) * nnz +
-                               sizeof(int32_t) * (size_t(pl->n_groups) + 1 + n_workers) + 16;
+    pl->n_ops = int(ops.size());
+    // tables of the staged encoder in shared memory: task records (32 bytes each), entry
+    // records, group records, TMA boxes
+    const size_t table_bytes = 32 * size_t(n_workers) + sizeof(AgcEntryDesc) * (size_t(nnz) + 1) +
+                               16 * size_t(pl->n_groups) + sizeof(AgcLoadOp) * ops.size() + 16;
     if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0 && table_bytes <= AGC_ENC_TABLE_BYTES_MAX) {
         const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16 + table_bytes;
         const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);  // two halves of max_rows x 1 KiB

@@ -296,6 +296,31 @@ def test_buckets_with_tiny_sums_of_squares(agc, torch, B, direct):
     assert (out["ghat"].view(np.uint32) == ref["ghat"].view(np.uint32)).all()
 
 
+@pytest.mark.parametrize("B,direct", [(512, False), (128, False), (512, True), (0, False), (2048, False)])
+def test_workers_without_entries_send_the_zero_vector(agc, torch, B, direct):
+    """A worker whose row of A is empty encodes f_i = 0: zero codes, scale 0, in every mode
+    (the unbiasedness check is off: the other workers carry the partitions)."""
+    rng = np.random.default_rng(5 + B)
+    n, k, d = 7, 5, 3 * 512 + 100
+    bits = np.array([3, 1, 8, 2, 5, 4, 6], np.uint8)
+    p = np.full(n, 0.2)
+    sup = [[0, 1], [], [2], [], [1, 3, 4], [0], []]
+    rp = np.zeros(n + 1, np.int32)
+    ci, a = [], []
+    for i, cols in enumerate(sup):
+        ci += cols
+        a += list(rng.uniform(0.3, 1.5, len(cols)))
+        rp[i + 1] = len(ci)
+    code = (rp, np.array(ci, np.int32), np.array(a, np.float32), rng.uniform(0.5, 1.5, n).astype(np.float32))
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    masks = np.ones((2, n), np.uint8)
+    masks[1, 2] = 0
+    out, ref = run_both(agc, torch, G, code, p, bits, B, 21, 2, masks,
+                        flags=agc.AGC_FLAG_FORCE_DIRECT if direct else 0)
+    assert_exact(out, ref)
+    assert (ref["scales"][[1, 3, 6]] == 0).all()
+
+
 def test_same_round_same_bits_other_round_other_bits(agc, torch):
     wl = cfgs.config1()
     code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
@@ -459,8 +484,7 @@ def test_encoder_division_is_correctly_rounded_everywhere(agc):
 
 
 def test_encoder_square_root_is_correctly_rounded_everywhere(agc):
-    """The encoder's branch-free square root against the IEEE one on its whole domain (every
-    float from 2^-102 up)."""
+    """The encoder's branch-free square root against the IEEE one for every normal float."""
     assert agc.agc_selftest_sqrt() == 0
 
 
