@@ -286,7 +286,8 @@ int agc_two_track_vector(int n, int k, const double *p, const uint8_t *bits, dou
  * launched), otherwise as agc_decode. Asynchronous on the stream.
  *
  * The first call on each device looks up the array's device address (with that device
- * current); make that first call outside any stream capture. All calls on a device
+ * current). Every call copies its tables from the host arrays given here, so a stream
+ * that is being captured is refused: AGC_ERR_STATE, nothing copied or launched. All calls on a device
  * share the one array: each call rewrites every entry it later reads, so nothing has
  * to be cleared between calls, but two calls whose GPU work overlaps (different
  * streams, or different threads) race on it - keep them on one stream or order them.
@@ -356,6 +357,31 @@ int agc_code_build(int n, int k, const double *p, const uint8_t *bits, double ph
                    double eta, int mode, const int32_t *sup_row_ptr,
                    const int32_t *sup_col_idx, int32_t nnz_cap, int32_t *row_ptr_out,
                    int32_t *col_out, float *a_out, float *w_out, double *Y_out);
+
+/*
+ * agc_bit_allocate_heuristic - the two heuristics that Sec. VI (Fig. 2) compares Algorithm 1
+ * and the exact DP with. The paper names them without printing them; the readings are:
+ *   AGC_ALLOC_GREEDY      the residual bits are handed out one at a time, each to the worker
+ *                         whose utility h_i of problem (b-SP1) gains most from it;
+ *   AGC_ALLOC_RELAXATION  the stationarity system of the continuous relaxation over all
+ *                         workers, rounded by floor + largest remainders (Algorithm 1's
+ *                         Lagrangian candidate without the search over the most reliable
+ *                         subsets, the equal split and the one-bit swaps).
+ * Arguments and errors as agc_bit_allocate. Host only.
+ */
+#define AGC_ALLOC_GREEDY 0
+#define AGC_ALLOC_RELAXATION 1
+int agc_bit_allocate_heuristic(int method, int n, const double *p, int Z_tot, int b_min, int b_max,
+                               double phi_dim, double eta, uint8_t *bits_out, double *F_out);
+/*
+ * agc_allocation_upper_bound - an upper bound on the optimum of problem (b-SP1) (Sec. III-B):
+ * each h_i is replaced by the upper concave envelope of its integer points, which makes the
+ * problem separable and concave; its optimum (the envelope's unit slopes, largest first) is
+ * written to *bound_out. F of the exact DP never exceeds it. Arguments and errors as
+ * agc_bit_allocate (no bits are returned). Host only.
+ */
+int agc_allocation_upper_bound(int n, const double *p, int Z_tot, int b_min, int b_max, double phi_dim,
+                               double eta, double *bound_out);
 
 /*
  * agc_eta_balance - the error-balance factor suggested in Sec. V-B:

@@ -399,6 +399,109 @@ def bit_allocate_bruteforce(p, z_tot, dim, b_max=0, eta=1.0):
     return (np.array(best_r) + 2).astype(np.uint8), float(best)
 
 
+# ---------------------------------------------------------------- comparison allocators (Sec. VI)
+# The paper's Fig. 2 sets Algorithm 1 against the exact DP and against two heuristics it names
+# without printing them, "greedy" and "continuous relaxation"; these are the readings taken.
+def bit_allocate_greedy(p, z_tot, dim, b_max=0, eta=1.0):
+    """Greedy heuristic: from r = 0, the residual bits are handed out one at a time, each to
+    the worker whose utility h_i gains most from one more bit (ties: lowest index). Exact when
+    every h_i is concave on the range; trapped by the convex foot of the sigmoidal h_i otherwise.
+    Returns (bits, F)."""
+    p = np.asarray(p, np.float64)
+    n = len(p)
+    z_res = int(z_tot) - 2 * n
+    assert z_res >= 0
+    cap = z_res if not b_max else min(z_res, b_max - 2)
+    assert n * cap >= z_res, "budget exceeds the cap"
+    hh = np.array([[h_utility(p[i], a, dim, eta) for a in range(cap + 2)] for i in range(n)])
+    r = np.zeros(n, np.int64)
+    idx = np.arange(n)
+    for _ in range(z_res):
+        gain = np.where(r < cap, hh[idx, np.minimum(r + 1, cap + 1)] - hh[idx, r], -np.inf)
+        r[int(np.argmax(gain))] += 1
+    return (r + 2).astype(np.uint8), float(hh[idx, r].sum())
+
+
+def bit_allocate_relaxation(p, z_tot, dim, b_max=0, eta=1.0):
+    """Continuous-relaxation heuristic: the stationarity system of the relaxed problem over ALL
+    workers (`_lagrangian_allocation` with every worker selected), rounded by floor + largest
+    remainders. It is Algorithm 1's LAG candidate without the search over the top-kappa sets,
+    the EQ candidate and the swap refinement. Returns (bits, F)."""
+    p = np.asarray(p, np.float64)
+    n = len(p)
+    z_res = int(z_tot) - 2 * n
+    assert z_res >= 0
+    cap = z_res if not b_max else min(z_res, b_max - 2)
+    assert n * cap >= z_res, "budget exceeds the cap"
+    if z_res == 0:
+        r = np.zeros(n, np.int64)
+    else:
+        r = _lagrangian_allocation(p, z_res, cap, dim, eta)
+        if r is None:   # rounding could not place the bits under the cap: spread them evenly
+            r = np.full(n, z_res // n, np.int64)
+            r[:z_res % n] += 1
+    return (r + 2).astype(np.uint8), allocation_value(p, r, dim, eta)
+
+
+def allocation_upper_bound(p, z_tot, dim, b_max=0, eta=1.0):
+    """An upper bound on the optimum of (b-SP1): each h_i is replaced by the upper concave
+    envelope of its integer points, which makes the problem a separable concave one whose
+    optimum the greedy rule over the envelope's unit slopes attains exactly. F_DP <= bound."""
+    p = np.asarray(p, np.float64)
+    n = len(p)
+    z_res = int(z_tot) - 2 * n
+    cap = z_res if not b_max else min(z_res, b_max - 2)
+    slopes = []
+    base = 0.0
+    for i in range(n):
+        h = np.array([h_utility(p[i], a, dim, eta) for a in range(cap + 1)])
+        base += h[0]
+        hull = [0]                                    # upper hull of the points (a, h[a])
+        for a in range(1, cap + 1):
+            while len(hull) >= 2:
+                a0, a1 = hull[-2], hull[-1]
+                if (h[a1] - h[a0]) * (a - a0) <= (h[a] - h[a0]) * (a1 - a0):
+                    hull.pop()
+                else:
+                    break
+            hull.append(a)
+        for a0, a1 in zip(hull[:-1], hull[1:]):
+            slopes += [(h[a1] - h[a0]) / (a1 - a0)] * (a1 - a0)
+    slopes = np.sort(np.array(slopes))[::-1]
+    return float(base + slopes[:z_res].sum())
+
+
+def allocator_study(ns=(10, 50), multiples=(1, 2, 3, 4, 5), seeds=50, dim=512.0, b_max=0, with_eta=False,
+                    probs=None):
+    """Synthetic re-creation of the comparison of Fig. 2 (Sec. VI): mean objective F(r) of
+    Algorithm 1, the exact DP, the greedy and the continuous-relaxation heuristics, and the
+    concave-envelope upper bound, over `seeds` draws of the straggler probabilities for
+    Z_res = multiple * n residual bits. `probs(n, seed)` supplies the probabilities (the
+    caller passes the shifted-exponential model of Sec. V-A). with_eta applies the
+    error-balance factor of Sec. V-B to every method. Returns a list of rows (dicts)."""
+    rows = []
+    for n in ns:
+        for mult in multiples:
+            z_tot = 2 * n + mult * n
+            acc = {"alg1": 0.0, "dp": 0.0, "greedy": 0.0, "relaxation": 0.0, "bound": 0.0}
+            worst = 1.0
+            for seed in range(seeds):
+                p = probs(n, seed)
+                eta = eta_balance(p, z_tot, dim) if with_eta else 1.0
+                f_dp = bit_allocate_dp(p, z_tot, dim, b_max, eta)[1]
+                f_a = bit_allocate_low_complexity(p, z_tot, dim, b_max, eta)[1]
+                acc["dp"] += f_dp
+                acc["alg1"] += f_a
+                acc["greedy"] += bit_allocate_greedy(p, z_tot, dim, b_max, eta)[1]
+                acc["relaxation"] += bit_allocate_relaxation(p, z_tot, dim, b_max, eta)[1]
+                acc["bound"] += allocation_upper_bound(p, z_tot, dim, b_max, eta)
+                worst = min(worst, f_a / f_dp)
+            row = {"n": n, "z_res": mult * n, "eta": bool(with_eta), "alg1_min_ratio": worst}
+            row.update({k: v / seeds for k, v in acc.items()})
+            rows.append(row)
+    return rows
+
+
 def eta_balance(p, z_tot, dim):
     """eta = mean(p) * 4 (2^(Z_tot/n - 1) - 1)^2 / l (Sec. V-B)."""
     p = np.asarray(p, np.float64)

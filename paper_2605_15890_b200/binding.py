@@ -19,6 +19,8 @@ AGC_STATUS_NONFINITE = 1
 AGC_STATUS_TIMEOUT = 4
 AGC_CODE_INTERVAL = 0
 AGC_CODE_SUPPORT = 1
+AGC_ALLOC_GREEDY = 0
+AGC_ALLOC_RELAXATION = 1
 AGC_ERR_LIMIT = -10
 
 
@@ -89,6 +91,11 @@ def _load():
     L.agc_selftest_division.restype = C.c_int
     L.agc_selftest_sqrt.argtypes = [C.POINTER(C.c_ulonglong)]
     L.agc_selftest_sqrt.restype = C.c_int
+    L.agc_bit_allocate_heuristic.argtypes = [C.c_int, C.c_int, f64p, C.c_int, C.c_int, C.c_int, C.c_double, C.c_double,
+                                             u8p, f64p]
+    L.agc_bit_allocate_heuristic.restype = C.c_int
+    L.agc_allocation_upper_bound.argtypes = [C.c_int, f64p, C.c_int, C.c_int, C.c_int, C.c_double, C.c_double, f64p]
+    L.agc_allocation_upper_bound.restype = C.c_int
     L.agc_eta_balance.argtypes = [C.c_int, f64p, C.c_int, C.c_double, f64p]
     L.agc_eta_balance.restype = C.c_int
     L.agc_strerror.argtypes = [C.c_int]
@@ -289,6 +296,24 @@ def agc_bit_allocate(p, z_tot, b_min=2, b_max=8, phi_dim=512.0, eta=1.0):
 
 def agc_bit_allocate_dp(p, z_tot, b_min=2, b_max=8, phi_dim=512.0, eta=1.0):
     return _alloc(_lib.agc_bit_allocate_dp, p, z_tot, b_min, b_max, phi_dim, eta)
+
+
+def agc_bit_allocate_heuristic(method, p, z_tot, b_min=2, b_max=8, phi_dim=512.0, eta=1.0):
+    """The greedy (AGC_ALLOC_GREEDY) or continuous-relaxation (AGC_ALLOC_RELAXATION) heuristic of
+    the allocator comparison. Returns (bits uint8 [n], F)."""
+    p = _np(p, np.float64)
+    bits = np.zeros(len(p), np.uint8)
+    F = C.c_double(0.0)
+    _check(_lib.agc_bit_allocate_heuristic(method, len(p), _hp(p, C.c_double), z_tot, b_min, b_max, phi_dim, eta,
+                                           _hp(bits, C.c_uint8), C.byref(F)))
+    return bits, F.value
+
+
+def agc_allocation_upper_bound(p, z_tot, b_min=2, b_max=8, phi_dim=512.0, eta=1.0):
+    p = _np(p, np.float64)
+    bound = C.c_double(0.0)
+    _check(_lib.agc_allocation_upper_bound(len(p), _hp(p, C.c_double), z_tot, b_min, b_max, phi_dim, eta, C.byref(bound)))
+    return bound.value
 
 
 def agc_code_build(n, k, p, bits, phi_dim, eta=1.0, mode=AGC_CODE_INTERVAL, sup_row_ptr=None,

@@ -1216,10 +1216,15 @@ extern "C" int agc_decode_update_static(int n_workers, int64_t d, uint32_t bucke
     for (int i = 0; i < n_workers; ++i)
         if (bits[i] < 1 || bits[i] > 8) return AGC_ERR_BITS;
 
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // every call copies its tables from the caller's host arrays and from this function's
+    // stack: a stream that is being captured would record those addresses, so it is refused
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return AGC_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return AGC_ERR_STATE;
     AgcStaticScratch *sc = nullptr;
     const int rc = agc_static_scratch_address(&sc);
     if (rc != AGC_OK) return rc;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     const long long nblk = (d + AGC_BLOCK - 1) / AGC_BLOCK;
     long long word_off[AGC_STATIC_MAX_WORKERS + 1];

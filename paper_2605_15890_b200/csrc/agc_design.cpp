@@ -229,6 +229,75 @@ extern "C" int agc_bit_allocate(int n, const double *p, int Z_tot, int b_min, in
     return AGC_OK;
 }
 
+// The two heuristics the paper's Fig. 2 sets Algorithm 1 against (Sec. VI names them without
+// printing them; these are the readings taken) and an upper bound on the optimum.
+extern "C" int agc_bit_allocate_heuristic(int method, int n, const double *p, int Z_tot, int b_min, int b_max,
+                                          double phi_dim, double eta, uint8_t *bits_out, double *F_out)
+{
+    int z_res, cap;
+    if (method != AGC_ALLOC_GREEDY && method != AGC_ALLOC_RELAXATION) return AGC_ERR_ARG;
+    if (int e = check_alloc_args(n, p, Z_tot, b_min, b_max, phi_dim, eta, bits_out, &z_res, &cap)) return e;
+    Utility h(n, cap, p, phi_dim, eta);
+    std::vector<int> r(n, 0);
+    if (method == AGC_ALLOC_GREEDY) {
+        // one bit at a time to the worker that gains most from it (ties: lowest index)
+        for (int bit = 0; bit < z_res; ++bit) {
+            double best = -std::numeric_limits<double>::infinity();
+            int at = -1;
+            for (int i = 0; i < n; ++i) {
+                if (r[i] >= cap) continue;
+                const double g = h(i, r[i] + 1) - h(i, r[i]);
+                if (g > best) { best = g; at = i; }
+            }
+            ++r[at];
+        }
+    } else if (z_res > 0) {
+        // the relaxed problem's stationarity system over all workers, rounded
+        std::vector<double> pall(p, p + n);
+        if (!lagrangian_allocation(pall, z_res, cap, phi_dim, eta, r)) {
+            for (int i = 0; i < n; ++i) r[i] = z_res / n + (i < z_res % n ? 1 : 0);
+        }
+    }
+    for (int i = 0; i < n; ++i) bits_out[i] = uint8_t(r[i] + 2);
+    if (F_out) *F_out = h.total(r);
+    return AGC_OK;
+}
+
+extern "C" int agc_allocation_upper_bound(int n, const double *p, int Z_tot, int b_min, int b_max, double phi_dim,
+                                          double eta, double *bound_out)
+{
+    int z_res, cap;
+    uint8_t dummy = 0;
+    if (!bound_out) return AGC_ERR_ARG;
+    if (int e = check_alloc_args(n, p, Z_tot, b_min, b_max, phi_dim, eta, &dummy, &z_res, &cap)) return e;
+    Utility h(n, cap, p, phi_dim, eta);
+    // upper concave envelope of each worker's integer points; the envelope's unit slopes,
+    // largest first, solve the separable concave problem exactly
+    std::vector<double> slopes;
+    double base = 0.0;
+    for (int i = 0; i < n; ++i) {
+        base += h(i, 0);
+        std::vector<int> hull(1, 0);
+        for (int a = 1; a <= cap; ++a) {
+            while (hull.size() >= 2) {
+                const int a0 = hull[hull.size() - 2], a1 = hull.back();
+                if ((h(i, a1) - h(i, a0)) * (a - a0) <= (h(i, a) - h(i, a0)) * (a1 - a0)) hull.pop_back();
+                else break;
+            }
+            hull.push_back(a);
+        }
+        for (size_t t = 0; t + 1 < hull.size(); ++t) {
+            const int a0 = hull[t], a1 = hull[t + 1];
+            for (int u = a0; u < a1; ++u) slopes.push_back((h(i, a1) - h(i, a0)) / (a1 - a0));
+        }
+    }
+    std::sort(slopes.begin(), slopes.end(), [](double x, double y) { return x > y; });
+    double bound = base;
+    for (int t = 0; t < z_res && t < int(slopes.size()); ++t) bound += slopes[t];
+    *bound_out = bound;
+    return AGC_OK;
+}
+
 extern "C" int agc_code_build(int n, int k, const double *p, const uint8_t *bits, double phi_dim,
                               double eta, int mode, const int32_t *sup_row_ptr,
                               const int32_t *sup_col_idx, int32_t nnz_cap, int32_t *row_ptr_out,

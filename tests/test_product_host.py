@@ -174,3 +174,30 @@ def test_allocator_under_the_papers_delay_model(n):
         r_eq = np.zeros(n, int)
         r_eq[order] = base + (np.arange(n) < rem)
         assert F >= od.allocation_value(p, r_eq, 512) * (1 - 1e-12)
+
+
+def test_comparison_allocators_against_oracle_and_orderings():
+    """The library's greedy / continuous-relaxation heuristics and its upper bound against the
+    oracle's (same readings, float64), and the orderings of the allocator comparison of Sec. VI on
+    the shifted-exponential model at n = 10 and 50."""
+    from paper_2605_15890_b200 import allocator_study
+    rng = np.random.default_rng(51)
+    for trial in range(6):
+        n = int(rng.integers(3, 14))
+        zres = int(rng.integers(1, 4 * n))
+        p = rng.uniform(0.02, 0.9, n)
+        dim = float(rng.choice([8, 512, 4096]))
+        z_tot = 2 * n + zres
+        bg, Fg = agc.agc_bit_allocate_heuristic(agc.AGC_ALLOC_GREEDY, p, z_tot, b_max=0, phi_dim=dim)
+        obg, oFg = od.bit_allocate_greedy(p, z_tot, dim)
+        assert (bg == obg).all() and np.isclose(Fg, oFg, rtol=1e-12)
+        br, Fr = agc.agc_bit_allocate_heuristic(agc.AGC_ALLOC_RELAXATION, p, z_tot, b_max=0, phi_dim=dim)
+        obr, oFr = od.bit_allocate_relaxation(p, z_tot, dim)
+        assert br.sum() == z_tot and np.isclose(Fr, oFr, rtol=1e-9)
+        assert np.isclose(agc.agc_allocation_upper_bound(p, z_tot, b_max=0, phi_dim=dim),
+                          od.allocation_upper_bound(p, z_tot, dim), rtol=1e-12)
+    for with_eta in (False, True):
+        for r in allocator_study.study(ns=(10, 50), multiples=(1, 3, 5), seeds=3, with_eta=with_eta):
+            assert r["alg1_min_ratio"] >= 0.99 and r["alg1"] <= r["dp"] * (1 + 1e-12)
+            assert r["greedy"] <= r["dp"] * (1 + 1e-12) and r["relaxation"] <= r["dp"] * (1 + 1e-12)
+            assert r["bound"] >= r["dp"] * (1 - 1e-12)

@@ -6,7 +6,7 @@ receives buffers): it keeps its working data in a fixed array inside the library
 of in a plan. Here it is called through the C ABI twice in a row, with different sizes,
 masks and learning rates the second time, so that anything an earlier call left in the
 shared array would show; each result must match what agc_decode gives for the same
-messages. The file name sorts last on purpose: with `-x` every other test has already run.
+messages, and what the CPU oracle gives when it applies the R updates one after the other. The file name sorts last on purpose: with `-x` every other test has already run.
 """
 import numpy as np
 import pytest
@@ -35,9 +35,15 @@ def _one_case(agc, torch, n, d, B, R, seed):
     agc.agc_decode_update_static(n, d, B, bits, w, ses.codes, ses.scales, masks, R, lr, got)
     torch.cuda.synchronize()
     want, got = want.cpu().numpy(), got.cpu().numpy()
+    codes, scales = ses.codes_host(), ses.scales_host()
     ses.close()
     assert np.abs(want - beta0).max() > 0                     # the update did something
     rel = np.abs(got - want).max() / np.abs(want).max()
+    assert rel <= 1e-5, rel
+    # and against the oracle's defining order: R updates one after the other
+    from oracle import roundpath as orp
+    _, ob = orp.decode(d, bits, B, w, masks.cpu().numpy(), codes, scales, lr=lr, beta=beta0, want_ghat=False)
+    rel = np.abs(got - ob).max() / np.abs(ob).max()
     assert rel <= 1e-5, rel
 
 
