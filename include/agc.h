@@ -115,11 +115,16 @@ size_t agc_worker_offset(const agc_plan_t *plan, int i);
  * The random draw of the stochastic rounding (Eq. rv_quant) is keyed by the position of
  * a coordinate in the worker's message. A plan that covers coordinates
  * [512 * first_block, 512 * first_block + d) of a longer gradient - one shard of it on
- * one GPU - then draws exactly what a plan over the whole vector draws there, and since
- * every bucket has its own norm, the shard's codes and scales are the corresponding
- * slices of the whole vector's. Default 0. first_block >= 0, first_block + ceil(d/512)
- * <= 2^26, and a multiple of bucket / 512 for buckets of 1024 and above (a range starts at
- * a bucket). Takes effect from the next agc_encode_quantize.
+ * one GPU - then draws exactly what a plan over the whole vector draws there. With
+ * bucket-wise norms every bucket has its own norm, so the shard's codes and scales are the
+ * corresponding slices of the whole vector's and agc_encode_quantize needs nothing else.
+ * With the global norm (bucket 0) the norm of Eq. quant_def is the whole vector's:
+ * agc_encode_quantize, agc_encode_quantize_rows and agc_round_host return AGC_ERR_STATE on
+ * such a plan once first_block != 0, and the shard is encoded with agc_encode_norm_sums,
+ * an exchange of n floats between the shards, and agc_encode_quantize_with_norms.
+ * Default 0. first_block >= 0, first_block + ceil(d/512) <= 2^26, and a multiple of
+ * bucket / 512 for buckets of 1024 and above (a range starts at a bucket). Takes effect from
+ * the next encode call.
  */
 int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block);
 /* 1 if the plan encodes with the TMA-staged kernel, 0 if with the direct-load kernel. */
@@ -143,6 +148,33 @@ int agc_plan_uses_tma(const agc_plan_t *plan);
 int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
                         void *codes_dev, float *scales_dev, uint32_t *status_dev,
                         void *cuda_stream);
+
+/*
+ * The global norm of Eq. quant_def (Sec. II-B: one l2 norm ||f_i||_2 per worker) for a vector
+ * that is split into contiguous ranges of pack blocks over several plans / GPUs. Three steps:
+ *
+ * agc_encode_norm_sums - first pass over this plan's coordinates: sumsq_dev[i] (device, n
+ *   floats) = sum of squares of worker i's coded vector over the plan's range, summed as the
+ *   single-call encoder sums it (512-coordinate block sums, then the pairwise tree over the
+ *   block sums in block order). Asynchronous on the stream.
+ * agc_combine_norm_sums - host helper for the exchange: per_range holds the ranges' sums in
+ *   range order (ranges x n floats, e.g. after an all-gather); the same pairwise tree continues
+ *   over them. When every range but the last covers the same power-of-two number of pack
+ *   blocks, each range's sum is a node of the whole vector's tree and the result - hence
+ *   every code and scale of step three - equals the unsplit encoder's bit for bit; any other
+ *   split adds the same squares in another order (a difference in the last bits of the norm).
+ * agc_encode_quantize_with_norms - second pass: encodes the plan's range with the norms
+ *   sqrt(sumsq_dev[i]) of the WHOLE vector (device, n floats, the combined sums) and the random
+ *   stream positions given by agc_plan_set_first_block. Writes the plan's codes and the n
+ *   scales (the same on every shard). Other arguments as agc_encode_quantize.
+ *
+ * All three return AGC_ERR_STATE for a plan that was not created with bucket 0.
+ */
+int agc_encode_norm_sums(agc_plan_t *plan, const float *G_dev, int64_t ld, float *sumsq_dev, void *cuda_stream);
+int agc_combine_norm_sums(int ranges, int n, const float *per_range, float *sumsq_out);
+int agc_encode_quantize_with_norms(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
+                                   const float *sumsq_dev, void *codes_dev, float *scales_dev,
+                                   uint32_t *status_dev, void *cuda_stream);
 
 /*
  * agc_encode_quantize_rows - the same round for partial gradients that live in k separate

@@ -395,26 +395,87 @@ void agc_oracle_adam_two_track(int64_t d, const float *gw, const float *gv, floa
  * the pairwise tree in block order, level by level: entry t of the next level is
  * v[2t] + v[2t+1], a last entry without partner is added to +0 (the same as a balanced tree
  * over the sums padded with +0 to a power of two). */
+/* the pairwise tree over len values in index order, level by level, in place; returns v[0] */
+static float shrinking_tree(float *v, int64_t len)
+{
+    while (len > 1) {
+        int64_t half = (len + 1) / 2;
+        for (int64_t t = 0; t < half; ++t)
+            v[t] = v[2 * t] + (2 * t + 1 < len ? v[2 * t + 1] : 0.0f);
+        len = half;
+    }
+    return v[0];
+}
+
 /*
- * Encode + quantise + pack with the global norm. Same wire format as the bucketed path;
- * scales has ONE entry per worker. A worker whose sum of squares is below the smallest
- * normal number or not finite is sent as zero codes with scale 0.
+ * Step 1 of the global norm: sumsq[i] = sum of squares of worker i's coded vector f_i over the
+ * d coordinates given (a whole vector, or one contiguous range of pack blocks of it), in the
+ * order stated above.
  */
-uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_t *row_ptr,
-                                           const int32_t *col_idx, const float *a,
-                                           const uint8_t *bits, uint64_t seed, uint64_t round,
-                                           const float *G, int64_t ld, uint32_t *codes,
-                                           float *scales, float *x_out)
+void agc_oracle_global_sumsq(int n, int k, int64_t d, const int32_t *row_ptr, const int32_t *col_idx,
+                             const float *a, const float *G, int64_t ld, float *sumsq)
+{
+    const int64_t nblk = agc_oracle_num_blocks(d);
+    float *x = (float *)malloc((size_t)AGC_BLOCK * sizeof(float));
+    float *part = (float *)malloc((size_t)nblk * sizeof(float));
+    (void)k;
+    for (int i = 0; i < n; ++i) {
+        for (int64_t q = 0; q < nblk; ++q) {
+            /* Sec. II-A: f_i, ascending partitions, fp32 fma chain; zero beyond d */
+            for (int o = 0; o < AGC_BLOCK; ++o) {
+                int64_t m = q * AGC_BLOCK + o;
+                float acc = 0.0f;
+                if (m < d)
+                    for (int e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                        acc = fmaf(a[e], G[(int64_t)col_idx[e] * ld + m], acc);
+                x[o] = acc;
+            }
+            part[q] = bucket_sumsq(x, AGC_BLOCK);
+        }
+        sumsq[i] = shrinking_tree(part, nblk);
+    }
+    free(x); free(part);
+}
+
+/*
+ * Sums of squares of several contiguous ranges of one vector combined into the whole vector's:
+ * the same pairwise tree, continued over the ranges' sums in range order. per_range is
+ * ranges x n. When every range but the last covers the same power-of-two number of pack
+ * blocks, each range's sum is a node of the whole vector's tree and the result equals the
+ * unsplit sum bit for bit; for other splits it is the same sum in another order.
+ */
+void agc_oracle_combine_sumsq(int ranges, int n, const float *per_range, float *sumsq)
+{
+    float *v = (float *)malloc((size_t)ranges * sizeof(float));
+    for (int i = 0; i < n; ++i) {
+        for (int r = 0; r < ranges; ++r) v[r] = per_range[(int64_t)r * n + i];
+        sumsq[i] = shrinking_tree(v, ranges);
+    }
+    free(v);
+}
+
+/*
+ * Step 2 of the global norm: encode + quantise + pack the d coordinates given with the norm
+ * sqrt(sumsq[i]) of worker i (Eq. quant_def; the sum is the WHOLE vector's even when the
+ * coordinates are a range of it that starts at pack block first_block: the random draws are
+ * keyed by the position in the whole message). scales has ONE entry per worker. A worker
+ * whose sum of squares is below the smallest normal number or not finite is sent as zero
+ * codes with scale 0.
+ */
+uint32_t agc_oracle_encode_quantize_with_norm(int n, int k, int64_t d, const int32_t *row_ptr,
+                                              const int32_t *col_idx, const float *a,
+                                              const uint8_t *bits, uint64_t seed, uint64_t round,
+                                              int64_t first_block, const float *G, int64_t ld,
+                                              const float *sumsq_all, uint32_t *codes, float *scales,
+                                              float *x_out)
 {
     const int64_t nblk = agc_oracle_num_blocks(d);
     uint32_t status = 0;
     float *x = (float *)malloc((size_t)nblk * AGC_BLOCK * sizeof(float));
-    float *part = (float *)malloc((size_t)nblk * sizeof(float));
     int64_t woff = 0;
     (void)k;
     for (int i = 0; i < n; ++i) {
         const int b = bits[i];
-        /* Sec. II-A: f_i, ascending partitions, fp32 fma chain; zero beyond d */
         for (int64_t m = 0; m < nblk * AGC_BLOCK; ++m) {
             float acc = 0.0f;
             if (m < d)
@@ -423,16 +484,7 @@ uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_
             x[m] = acc;
         }
         if (x_out) memcpy(x_out + (int64_t)i * d, x, (size_t)d * sizeof(float));
-        for (int64_t q = 0; q < nblk; ++q) part[q] = bucket_sumsq(x + q * AGC_BLOCK, AGC_BLOCK);
-        /* shrinking tree: level by level over the current length */
-        int64_t len = nblk;
-        while (len > 1) {
-            int64_t half = (len + 1) / 2;
-            for (int64_t t = 0; t < half; ++t)
-                part[t] = part[2 * t] + (2 * t + 1 < len ? part[2 * t + 1] : 0.0f);
-            len = half;
-        }
-        float sumsq = part[0];
+        float sumsq = sumsq_all[i];
         int finite = (sumsq == sumsq) && (sumsq != INFINITY);
         int flushed = !(finite && sumsq >= 1.17549435e-38f);
         if (!finite) status |= AGC_ORACLE_STATUS_NONFINITE;
@@ -449,7 +501,7 @@ uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_
                     code = zero_code(b);
                 } else {
                     uint32_t u = agc_oracle_uniform15(seed, round, (uint32_t)i,
-                                                      (uint64_t)q * AGC_BLOCK + (uint64_t)pos);
+                                                      (uint64_t)(q + first_block) * AGC_BLOCK + (uint64_t)pos);
                     code = agc_oracle_quantize_one(x[q * AGC_BLOCK + o], inv, b, u);
                     if (code > 2u * zero_code(b) + (b == 1 ? 1u : 0u)) status |= AGC_ORACLE_STATUS_RANGE;
                     code &= (1u << b) - 1u;
@@ -461,7 +513,25 @@ uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_
             }
         woff += nblk * 16 * b;
     }
-    free(x); free(part);
+    free(x);
+    return status;
+}
+
+/*
+ * Encode + quantise + pack a whole vector with the global norm: step 1, then step 2. Same wire
+ * format as the bucketed path.
+ */
+uint32_t agc_oracle_encode_quantize_global(int n, int k, int64_t d, const int32_t *row_ptr,
+                                           const int32_t *col_idx, const float *a,
+                                           const uint8_t *bits, uint64_t seed, uint64_t round,
+                                           const float *G, int64_t ld, uint32_t *codes,
+                                           float *scales, float *x_out)
+{
+    float *sumsq = (float *)malloc((size_t)n * sizeof(float));
+    agc_oracle_global_sumsq(n, k, d, row_ptr, col_idx, a, G, ld, sumsq);
+    uint32_t status = agc_oracle_encode_quantize_with_norm(n, k, d, row_ptr, col_idx, a, bits, seed, round, 0, G, ld,
+                                                           sumsq, codes, scales, x_out);
+    free(sumsq);
     return status;
 }
 

@@ -52,6 +52,13 @@ def lib():
         L.agc_oracle_encode_quantize_global.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_uint64,
                                                         C.c_uint64, f32p, C.c_int64, u32p, f32p, f32p]
         L.agc_oracle_encode_quantize_global.restype = C.c_uint32
+        L.agc_oracle_global_sumsq.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, f32p, C.c_int64, f32p]
+        L.agc_oracle_global_sumsq.restype = None
+        L.agc_oracle_combine_sumsq.argtypes = [C.c_int, C.c_int, f32p, f32p]
+        L.agc_oracle_combine_sumsq.restype = None
+        L.agc_oracle_encode_quantize_with_norm.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_uint64,
+                                                           C.c_uint64, C.c_int64, f32p, C.c_int64, f32p, u32p, f32p, f32p]
+        L.agc_oracle_encode_quantize_with_norm.restype = C.c_uint32
         L.agc_oracle_encode_quantize_grouped.argtypes = [C.c_int, C.c_int, C.c_int64, i32p, i32p, f32p, u8p, C.c_int64,
                                                          C.c_uint64, C.c_uint64, f32p, C.c_int64, u32p, f32p, f32p]
         L.agc_oracle_encode_quantize_grouped.restype = C.c_uint32
@@ -240,6 +247,47 @@ def encode_quantize_global(row_ptr, col_idx, a, bits, seed, rnd, G, d=None, want
                                                  _p(G, C.c_float), ld, _p(codes, C.c_uint32),
                                                  _p(scales, C.c_float), _p(x, C.c_float))
     return codes, scales, int(st), x
+
+
+def global_sumsq(row_ptr, col_idx, a, G, d=None):
+    """Step 1 of the global norm: per-worker sum of squares of the coded vector over the
+    coordinates given (a whole vector or a contiguous range of pack blocks). float32 [n]."""
+    G = np.asarray(G)
+    assert G.dtype == np.float32 and G.ndim == 2 and G.strides[1] == 4
+    d = G.shape[1] if d is None else d
+    row_ptr, col_idx, a = _c(row_ptr, np.int32), _c(col_idx, np.int32), _c(a, np.float32)
+    n = len(row_ptr) - 1
+    out = np.zeros(n, np.float32)
+    lib().agc_oracle_global_sumsq(n, G.shape[0], d, _p(row_ptr, C.c_int32), _p(col_idx, C.c_int32), _p(a, C.c_float),
+                                  _p(G, C.c_float), G.strides[0] // 4, _p(out, C.c_float))
+    return out
+
+
+def combine_sumsq(per_range):
+    """Sums of squares of consecutive ranges, (ranges, n), combined into the whole vector's."""
+    per_range = _c(np.atleast_2d(per_range), np.float32)
+    out = np.zeros(per_range.shape[1], np.float32)
+    lib().agc_oracle_combine_sumsq(per_range.shape[0], per_range.shape[1], _p(per_range, C.c_float), _p(out, C.c_float))
+    return out
+
+
+def encode_quantize_with_norm(row_ptr, col_idx, a, bits, seed, rnd, G, sumsq, first_block=0, d=None):
+    """Step 2 of the global norm on the coordinates given, with the whole vector's sums of
+    squares. Returns (codes uint32, scales float32 [n], status)."""
+    G = np.asarray(G)
+    assert G.dtype == np.float32 and G.ndim == 2 and G.strides[1] == 4
+    d = G.shape[1] if d is None else d
+    row_ptr, col_idx = _c(row_ptr, np.int32), _c(col_idx, np.int32)
+    a, bits, sumsq = _c(a, np.float32), _c(bits, np.uint8), _c(sumsq, np.float32)
+    n = len(bits)
+    off = worker_word_offsets(d, bits)
+    codes = np.zeros(int(off[-1]), np.uint32)
+    scales = np.zeros(n, np.float32)
+    st = lib().agc_oracle_encode_quantize_with_norm(n, G.shape[0], d, _p(row_ptr, C.c_int32), _p(col_idx, C.c_int32),
+                                                    _p(a, C.c_float), _p(bits, C.c_uint8), seed, rnd, first_block,
+                                                    _p(G, C.c_float), G.strides[0] // 4, _p(sumsq, C.c_float),
+                                                    _p(codes, C.c_uint32), _p(scales, C.c_float), None)
+    return codes, scales, int(st)
 
 
 def encode_quantize_grouped(row_ptr, col_idx, a, bits, B, seed, rnd, G, d=None, want_x=False):

@@ -66,6 +66,12 @@ def _load():
     L.agc_encode_quantize.restype = C.c_int
     L.agc_encode_quantize_rows.argtypes = [vp, vp, C.c_uint64, vp, vp, vp, vp]
     L.agc_encode_quantize_rows.restype = C.c_int
+    L.agc_encode_norm_sums.argtypes = [vp, vp, C.c_int64, vp, vp]
+    L.agc_encode_norm_sums.restype = C.c_int
+    L.agc_combine_norm_sums.argtypes = [C.c_int, C.c_int, f32p, f32p]
+    L.agc_combine_norm_sums.restype = C.c_int
+    L.agc_encode_quantize_with_norms.argtypes = [vp, vp, C.c_int64, C.c_uint64, vp, vp, vp, vp, vp]
+    L.agc_encode_quantize_with_norms.restype = C.c_int
     L.agc_decode.argtypes = [vp, vp, vp, vp, C.c_int, f32p, vp, vp, vp, vp]
     L.agc_decode.restype = C.c_int
     L.agc_decode_update_static.argtypes = [C.c_int, C.c_int64, C.c_uint32, u8p, f32p, vp, vp, vp, C.c_int, f32p,
@@ -194,6 +200,27 @@ def agc_encode_quantize_rows(plan, G_rows_dev, rnd, codes_dev, scales_dev, statu
     """G_rows_dev: device array of k row addresses (a torch int64 CUDA tensor)."""
     _check(_lib.agc_encode_quantize_rows(plan, _dev(G_rows_dev), rnd, _dev(codes_dev), _dev(scales_dev),
                                          _dev(status_dev), _stream(stream)))
+
+
+def agc_encode_norm_sums(plan, G_dev, ld, sumsq_dev, stream=None):
+    """First pass of the global-norm encoder over the plan's coordinates: n sums of squares."""
+    _check(_lib.agc_encode_norm_sums(plan, _dev(G_dev), ld, _dev(sumsq_dev), _stream(stream)))
+
+
+def agc_combine_norm_sums(per_range):
+    """per_range: (ranges, n) float32 host array in range order; returns the combined sums [n]."""
+    per_range = np.ascontiguousarray(np.atleast_2d(per_range), np.float32)
+    out = np.zeros(per_range.shape[1], np.float32)
+    _check(_lib.agc_combine_norm_sums(per_range.shape[0], per_range.shape[1], _hp(per_range, C.c_float),
+                                      _hp(out, C.c_float)))
+    return out
+
+
+def agc_encode_quantize_with_norms(plan, G_dev, ld, rnd, sumsq_dev, codes_dev, scales_dev, status_dev=None,
+                                   stream=None):
+    """Second pass of the global-norm encoder with the whole vector's sums of squares."""
+    _check(_lib.agc_encode_quantize_with_norms(plan, _dev(G_dev), ld, rnd, _dev(sumsq_dev), _dev(codes_dev),
+                                               _dev(scales_dev), _dev(status_dev), _stream(stream)))
 
 
 def agc_decode(plan, codes_dev, scales_dev, masks_dev, R, lr_host=None, ghat_dev=None, beta_dev=None,

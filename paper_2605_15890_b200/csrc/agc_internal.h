@@ -127,7 +127,7 @@ struct agc_plan {
     bool global_norm = false;     // one l2 norm per worker (bucket argument 0)
     int group_blocks = 0;         // pack blocks per bucket for bucket arguments 1024, 2048, 4096 (else 0)
     int scale_shift = 0;          // see AgcDecParams
-    float *d_partials = nullptr, *d_chunk_sums = nullptr, *d_ginv = nullptr;
+    float *d_partials = nullptr, *d_chunk_sums = nullptr, *d_ginv = nullptr, *d_sums = nullptr;
     uint32_t flags = 0;
     int device = 0, sm_count = 0;
     std::vector<int32_t> row_ptr, col_idx;
@@ -171,7 +171,8 @@ struct agc_plan {
 };
 
 int agc_launch_encode(agc_plan *plan, const float *G, const float *const *G_rows, long long ld, uint64_t round,
-                      void *codes, float *scales, uint32_t *status, cudaStream_t stream);
+                      void *codes, float *scales, uint32_t *status, cudaStream_t stream, const float *sums_in = nullptr,
+                      float *sums_out = nullptr);
 int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, const uint8_t *masks,
                       int R, const float *lr_host, float *ghat, float *beta, uint32_t *status,
                       cudaStream_t stream);

@@ -112,7 +112,7 @@ void free_device(agc_plan *p)
     cudaFree(p->d_bits); cudaFree(p->d_wdesc); cudaFree(p->d_edesc); cudaFree(p->d_word_off);
     cudaFree(p->d_grp_row_ptr); cudaFree(p->d_grp_op_ptr); cudaFree(p->d_ops); cudaFree(p->d_grp_wk_ptr); cudaFree(p->d_grp_workers);
     cudaFree(p->d_weff); cudaFree(p->d_lr); cudaFree(p->d_v);
-    cudaFree(p->d_partials); cudaFree(p->d_chunk_sums); cudaFree(p->d_ginv);
+    cudaFree(p->d_partials); cudaFree(p->d_chunk_sums); cudaFree(p->d_ginv); cudaFree(p->d_sums);
     cudaFree(p->h_G); cudaFree(p->h_ghat); cudaFree(p->h_scales); cudaFree(p->h_codes);
     cudaFree(p->h_mask); cudaFree(p->h_status);
 }
@@ -249,7 +249,8 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
         const size_t nchunk = size_t((pl->nblk + 1023) / 1024);
         if (cudaMalloc(reinterpret_cast<void **>(&pl->d_partials), sizeof(float) * size_t(n_workers) * size_t(pl->nblk)) != cudaSuccess ||
             cudaMalloc(reinterpret_cast<void **>(&pl->d_chunk_sums), sizeof(float) * size_t(n_workers) * nchunk) != cudaSuccess ||
-            cudaMalloc(reinterpret_cast<void **>(&pl->d_ginv), sizeof(float) * size_t(n_workers) * size_t(pl->nb)) != cudaSuccess)
+            cudaMalloc(reinterpret_cast<void **>(&pl->d_ginv), sizeof(float) * size_t(n_workers) * size_t(pl->nb)) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void **>(&pl->d_sums), sizeof(float) * size_t(n_workers)) != cudaSuccess)
             rc = AGC_ERR_NOMEM;
     }
     if (!rc && cudaMalloc(reinterpret_cast<void **>(&pl->d_v), sizeof(float) * n_workers) != cudaSuccess) rc = AGC_ERR_NOMEM;
@@ -283,9 +284,6 @@ extern "C" int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block)
 {
     if (!plan || first_block < 0 || first_block + plan->nblk > (int64_t(1) << 26)) return AGC_ERR_ARG;
     if (plan->group_blocks && first_block % plan->group_blocks) return AGC_ERR_ARG;   // a range starts at a bucket
-    // one norm per worker over the WHOLE vector (Eq. quant_def): a range of it cannot be
-    // encoded on its own, its norm would be the range's
-    if (plan->global_norm && first_block != 0) return AGC_ERR_STATE;
     plan->first_block = first_block;
     return AGC_OK;
 }
@@ -299,8 +297,55 @@ extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t
     if ((ld & 3) || (reinterpret_cast<uintptr_t>(G_dev) & 15) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
         (reinterpret_cast<uintptr_t>(scales_dev) & 3))
         return AGC_ERR_ALIGN;
+    // one norm per worker over the WHOLE vector (Eq. quant_def): a range of a longer vector
+    // cannot be encoded on its own, its norm would be the range's
+    if (plan->global_norm && plan->first_block != 0) return AGC_ERR_STATE;
     return agc_launch_encode(plan, G_dev, nullptr, ld, round, codes_dev, scales_dev, status_dev,
                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int agc_encode_norm_sums(agc_plan_t *plan, const float *G_dev, int64_t ld, float *sumsq_dev, void *cuda_stream)
+{
+    if (!plan || !G_dev || !sumsq_dev || ld < plan->d) return AGC_ERR_ARG;
+    if (!plan->global_norm) return AGC_ERR_STATE;
+    if ((ld & 3) || (reinterpret_cast<uintptr_t>(G_dev) & 15) || (reinterpret_cast<uintptr_t>(sumsq_dev) & 3)) return AGC_ERR_ALIGN;
+    return agc_launch_encode(plan, G_dev, nullptr, ld, 0, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream),
+                             nullptr, sumsq_dev);
+}
+
+extern "C" int agc_encode_quantize_with_norms(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
+                                              const float *sumsq_dev, void *codes_dev, float *scales_dev,
+                                              uint32_t *status_dev, void *cuda_stream)
+{
+    if (!plan || !G_dev || !sumsq_dev || !codes_dev || !scales_dev || ld < plan->d) return AGC_ERR_ARG;
+    if (!plan->global_norm) return AGC_ERR_STATE;
+    if ((ld & 3) || (reinterpret_cast<uintptr_t>(G_dev) & 15) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
+        (reinterpret_cast<uintptr_t>(scales_dev) & 3) || (reinterpret_cast<uintptr_t>(sumsq_dev) & 3))
+        return AGC_ERR_ALIGN;
+    return agc_launch_encode(plan, G_dev, nullptr, ld, round, codes_dev, scales_dev, status_dev,
+                             static_cast<cudaStream_t>(cuda_stream), sumsq_dev, nullptr);
+}
+
+// Sums of squares of consecutive ranges of one vector, ranges x n on the host, combined by the
+// pairwise tree in range order (a last entry without partner is added to +0).
+extern "C" int agc_combine_norm_sums(int ranges, int n, const float *per_range, float *sumsq_out)
+{
+    if (ranges < 1 || n < 1 || !per_range || !sumsq_out) return AGC_ERR_ARG;
+    std::vector<float> v(ranges);
+    for (int i = 0; i < n; ++i) {
+        for (int r = 0; r < ranges; ++r) v[r] = per_range[size_t(r) * n + i];
+        int len = ranges;
+        while (len > 1) {
+            const int half = (len + 1) / 2;
+            for (int t = 0; t < half; ++t) {
+                volatile float sum = v[2 * t] + (2 * t + 1 < len ? v[2 * t + 1] : 0.0f);   // one fp32 addition
+                v[t] = sum;
+            }
+            len = half;
+        }
+        sumsq_out[i] = v[0];
+    }
+    return AGC_OK;
 }
 
 extern "C" int agc_encode_quantize_rows(agc_plan_t *plan, const float *const *G_rows_dev, uint64_t round,
@@ -311,6 +356,7 @@ extern "C" int agc_encode_quantize_rows(agc_plan_t *plan, const float *const *G_
     if ((reinterpret_cast<uintptr_t>(G_rows_dev) & 7) || (reinterpret_cast<uintptr_t>(codes_dev) & 15) ||
         (reinterpret_cast<uintptr_t>(scales_dev) & 3))
         return AGC_ERR_ALIGN;
+    if (plan->global_norm && plan->first_block != 0) return AGC_ERR_STATE;
     return agc_launch_encode(plan, nullptr, G_rows_dev, 0, round, codes_dev, scales_dev, status_dev,
                              static_cast<cudaStream_t>(cuda_stream));
 }
@@ -364,6 +410,7 @@ extern "C" int agc_round_host(agc_plan_t *plan, const float *G_host, int64_t ld_
                               void *cuda_stream)
 {
     if (!plan || !G_host || !mask_host || !ghat_host || ld_host < plan->d) return AGC_ERR_ARG;
+    if (plan->global_norm && plan->first_block != 0) return AGC_ERR_STATE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const long long ld_dev = (plan->d + 3) & ~3LL;
     if (!plan->h_G) {

@@ -400,6 +400,60 @@ def test_shards_with_block_offsets_reproduce_the_whole_vector(agc, torch):
         ses.close()
 
 
+@pytest.mark.parametrize("d,shards,direct", [(512 * 11 + 37, 3, False), (600_001, 2, False), (512 * 11 + 37, 2, True)])
+def test_global_norm_over_shards_equals_the_whole_vector(agc, torch, d, shards, direct):
+    """One norm per worker over a vector held as `shards` plans (one GPU here, one per GPU in
+    use): first pass per shard, the library's combine of the shards' sums, second pass with the
+    whole vector's sums and the shard's block offset. With power-of-two shard sizes the
+    codes and scales equal the oracle's unsplit global-norm encoding bit for bit; a plain
+    agc_encode_quantize on an offset global-norm plan is refused."""
+    from paper_2605_15890_b200 import sharding
+    from paper_2605_15890_b200.session import Session
+    rng = np.random.default_rng(d)
+    n, k = 5, 6
+    bits = np.array([2, 3, 8, 1, 6], np.uint8)
+    p = rng.uniform(0.05, 0.4, n)
+    rp, ci, a, w = _codes.cyclic_code(p, bits, k, 3, 512)
+    G_host = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 2, (k, 1))).astype(np.float32)
+    oc, osc, ost, _ = orp.encode_quantize_global(rp, ci, a, bits, 31, 7, G_host)
+    off = orp.worker_word_offsets(d, bits)
+    flags = agc.AGC_FLAG_ALLOW_1BIT | (agc.AGC_FLAG_FORCE_DIRECT if direct else 0)
+    parts = []
+    for r in range(shards):
+        lo, hi = sharding.power_of_two_range(d, r, shards)
+        assert hi > lo
+        ses = Session(n, k, hi - lo, rp, ci, a, w, p, bits, bucket=0, seed=31, flags=flags)
+        ses.set_first_block(lo // 512)
+        ld = (hi - lo + 3) // 4 * 4
+        Gd = torch.zeros((k, ld), dtype=torch.float32, device="cuda")
+        Gd[:, :hi - lo] = torch.from_numpy(G_host[:, lo:hi])
+        sums = torch.empty(n, dtype=torch.float32, device="cuda")
+        agc.agc_encode_norm_sums(ses.plan, Gd, ld, sums)
+        parts.append(dict(lo=lo, hi=hi, ses=ses, G=Gd, ld=ld, sums=sums))
+    if shards > 1:
+        with pytest.raises(agc.AgcError):
+            parts[1]["ses"].encode(parts[1]["G"], 7)
+    torch.cuda.synchronize()
+    whole = agc.agc_combine_norm_sums(np.stack([pt["sums"].cpu().numpy() for pt in parts]))
+    assert (whole.view(np.uint32) == orp.global_sumsq(rp, ci, a, G_host).view(np.uint32)).all()
+    whole_dev = torch.from_numpy(whole).cuda()
+    for pt in parts:
+        ses = pt["ses"]
+        ses.codes.fill_(-1)
+        agc.agc_encode_quantize_with_norms(ses.plan, pt["G"], pt["ld"], 7, whole_dev, ses.codes, ses.scales, ses.status)
+        torch.cuda.synchronize()
+        assert int(ses.status.item()) == 0 and ost == 0
+        assert (ses.scales.cpu().numpy().view(np.uint32) == osc.view(np.uint32)).all()
+        got = ses.codes_host()
+        roff = orp.worker_word_offsets(pt["hi"] - pt["lo"], bits)
+        q0, nq = pt["lo"] // 512, (pt["hi"] - pt["lo"] + 511) // 512
+        for i in range(n):
+            b = int(bits[i])
+            want = oc[off[i] + q0 * 16 * b: off[i] + (q0 + nq) * 16 * b]
+            assert (got[roff[i]:roff[i + 1]] == want).all(), (pt["lo"], i)
+        ses.close()
+
+
 def test_config5_shape_one_bit_workers_and_64_realisations(agc, torch):
     """cfg5's structure at a size the oracle finishes: n=k=100, s=5, Student-t(3) values,
     bits 1..8, 64 realisations decoded per encode with the update fused."""

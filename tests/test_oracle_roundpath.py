@@ -702,3 +702,53 @@ def test_grouped_bucket_encoder_pins():
         L = (1 << (int(bits[i]) - 1)) - 1
         sigma = np.repeat(per_block[i], 512)[:d] / L / 2.0 / np.sqrt(rounds)
         assert (np.abs(acc[i] / rounds - x[i]) <= 6.0 * sigma + 1e-12).all()
+
+
+def test_global_norm_split_into_ranges_pins():
+    """The global norm over a vector split into contiguous ranges of pack blocks: with every range
+    but the last a power-of-two number of blocks the combined sums, and hence every code and
+    scale, equal the unsplit encoder's bit for bit; the sums agree with float64; an uneven split
+    gives the same sum up to the order of additions; a changed value in one range changes the
+    codes of the others only through the norm."""
+    rng = np.random.default_rng(71)
+    n, k = 3, 4
+    d = 512 * 11 + 37                     # 12 pack blocks
+    rp = np.array([0, 2, 3, 5], np.int32)
+    ci = np.array([0, 1, 2, 1, 3], np.int32)
+    a = rng.uniform(0.2, 1.5, 5).astype(np.float32)
+    bits = np.array([2, 5, 8], np.uint8)
+    G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-2, 2, (k, 1))).astype(np.float32)
+    whole_c, whole_s, st, x = orp.encode_quantize_global(rp, ci, a, bits, 13, 2, G, want_x=True)
+    whole_sums = orp.global_sumsq(rp, ci, a, G)
+    ref64 = (x.astype(np.float64) ** 2).sum(axis=1)
+    assert np.allclose(whole_sums, ref64, rtol=2e-6)
+    assert (np.sqrt(whole_sums).astype(np.float32).view(np.uint32) == whole_s.view(np.uint32)).all()
+    off = orp.worker_word_offsets(d, bits)
+    for per in (4, 8):                    # blocks per range: powers of two -> ranges of 4,4,4 and 8,4
+        cuts = list(range(0, 12, per)) + [12]
+        sums = np.stack([orp.global_sumsq(rp, ci, a, np.ascontiguousarray(G[:, b0 * 512:min(b1 * 512, d)]))
+                         for b0, b1 in zip(cuts[:-1], cuts[1:])])
+        comb = orp.combine_sumsq(sums)
+        assert (comb.view(np.uint32) == whole_sums.view(np.uint32)).all()
+        for b0, b1 in zip(cuts[:-1], cuts[1:]):
+            Gr = np.ascontiguousarray(G[:, b0 * 512:min(b1 * 512, d)])
+            c, s, st = orp.encode_quantize_with_norm(rp, ci, a, bits, 13, 2, Gr, comb, first_block=b0)
+            assert st == 0 and (s.view(np.uint32) == whole_s.view(np.uint32)).all()
+            roff = orp.worker_word_offsets(Gr.shape[1], bits)
+            for i in range(n):
+                b = int(bits[i])
+                want = whole_c[off[i] + b0 * 16 * b: off[i] + b1 * 16 * b]
+                assert (c[roff[i]:roff[i + 1]] == want).all(), (per, b0, i)
+    # an uneven split (5 + 7 blocks): the same sum in another order
+    sums = np.stack([orp.global_sumsq(rp, ci, a, np.ascontiguousarray(G[:, :5 * 512])),
+                     orp.global_sumsq(rp, ci, a, np.ascontiguousarray(G[:, 5 * 512:]))])
+    comb = orp.combine_sumsq(sums)
+    assert np.allclose(comb, ref64, rtol=2e-6)
+    # the order is the pairwise tree: (r0 + r1) + (r2 + r3), a last range without partner + 0;
+    # values chosen so that left-to-right and right-to-left sums give another float
+    e = 2.0 ** -24
+    v = np.array([[e], [1.0], [e], [e]], np.float32)
+    assert orp.combine_sumsq(v)[0] == np.float32(1.0 + 2.0 ** -23)        # left to right: 1.0
+    v = np.array([[e], [e], [1.0]], np.float32)
+    assert orp.combine_sumsq(v)[0] == np.float32(1.0 + 2.0 ** -23)        # right to left: 1.0
+    assert orp.combine_sumsq(v[:1])[0] == np.float32(e)

@@ -87,6 +87,70 @@ def test_two_ranks_reproduce_the_whole_encoding(tmp_path):
     assert (tmp_path / "ok").exists()
 
 
+def _rank_main_global_norm(rank, world, port, out_dir):
+    """The global norm (one l2 norm per worker over the whole vector) on two ranks: first pass on
+    the rank's range, all-gather of n floats, the library's combine on every rank, second pass
+    with the whole vector's sums. Oracle arithmetic per range; the split, the exchange and the
+    combine are the product's."""
+    import paper_2605_15890_b200 as agc
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        n, k, d, bits, (rp, ci, a, w), G = _problem()
+        seed, rnd = 9, 4
+        lo, hi = sharding.power_of_two_range(d, rank, world)
+        Gr = np.ascontiguousarray(G[:, lo:hi])
+        local = orp.global_sumsq(rp, ci, a, Gr)
+        sums = sharding.global_norm_sums(torch.from_numpy(local), agc.agc_combine_norm_sums)
+        c, s, st = orp.encode_quantize_with_norm(rp, ci, a, bits, seed, rnd, Gr, sums, first_block=lo // 512)
+        assert st == 0
+        gathered = [None] * world
+        dist.all_gather_object(gathered, (lo, hi, c, s, sums))
+        if rank == 0:
+            whole_c, whole_s, st, _ = orp.encode_quantize_global(rp, ci, a, bits, seed, rnd, G)
+            off = orp.worker_word_offsets(d, bits)
+            prev = 0
+            for glo, ghi, gc, gs, gsums in gathered:
+                assert glo == prev and glo % 512 == 0
+                prev = ghi
+                assert (gsums.view(np.uint32) == gathered[0][4].view(np.uint32)).all()   # identical norms on all ranks
+                assert (gs.view(np.uint32) == whole_s.view(np.uint32)).all()
+                roff = orp.worker_word_offsets(ghi - glo, bits)
+                nb_r = (ghi - glo + 511) // 512
+                for i in range(n):
+                    b = int(bits[i])
+                    want = whole_c[off[i] + (glo // 512) * 16 * b: off[i] + (glo // 512 + nb_r) * 16 * b]
+                    assert (gc[roff[i]:roff[i + 1]] == want).all(), (glo, i)
+            assert prev == d
+            with open(os.path.join(out_dir, "ok_global"), "w") as fh:
+                fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_global_norm_with_one_exchange(tmp_path):
+    world = 2
+    mp.spawn(_rank_main_global_norm, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    assert (tmp_path / "ok_global").exists()
+
+
+@pytest.mark.parametrize("d,world", [(1, 2), (512 * 8, 2), (512 * 7 + 100, 2), (25_557_032, 8), (10**8, 3), (513, 4)])
+def test_power_of_two_ranges_tile_the_vector(d, world):
+    prev = 0
+    sizes = []
+    for r in range(world):
+        lo, hi = sharding.power_of_two_range(d, r, world)
+        assert lo == prev and lo <= hi <= d and (lo % 512 == 0 or lo == d)
+        sizes.append((hi - lo + 511) // 512)
+        prev = hi
+    assert prev == d
+    per = sizes[0]
+    assert per & (per - 1) == 0                      # a power of two
+    full = [s for s in sizes if s == per]
+    assert all(s <= per for s in sizes) and sizes[:len(full)] == full
+
+
 @pytest.mark.parametrize("d,world", [(0, 3), (1, 2), (511, 2), (512, 2), (513, 4), (25_557_032, 8), (10**8, 3)])
 def test_coordinate_ranges_tile_the_vector(d, world):
     prev = 0
