@@ -129,6 +129,15 @@ size_t agc_worker_offset(const agc_plan_t *plan, int i);
 int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block);
 /* 1 if the plan encodes with the TMA-staged kernel, 0 if with the direct-load kernel. */
 int agc_plan_uses_tma(const agc_plan_t *plan);
+/*
+ * agc_plan_encode_layout - how the staged encoder tiles the encode of Sec. II-A for this plan.
+ * out4 (host, 4 ints): [0] 1 = staged kernel, 0 = direct-load kernel (then the rest is 0);
+ * [1] worker groups per pack block; [2] partition rows brought into shared memory per pack
+ * block, all groups together (k when every partition row is staged exactly once; more when the
+ * supports of different groups share partitions, which are then read again through L2);
+ * [3] depth of the shared-memory ring.
+ */
+int agc_plan_encode_layout(const agc_plan_t *plan, int32_t *out4);
 
 /*
  * agc_encode_quantize - one round of all n workers: encode, quantise, pack.

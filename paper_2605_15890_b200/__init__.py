@@ -14,7 +14,7 @@ _BINDING_NAMES = (
     "AGC_FLAG_NO_UNBIASED_CHECK", "AGC_STATUS_NONFINITE", "AGC_STATUS_TIMEOUT", "AgcError",
     "AGC_ALLOC_GREEDY", "AGC_ALLOC_RELAXATION", "agc_allocation_upper_bound", "agc_bit_allocate", "agc_bit_allocate_dp", "agc_bit_allocate_heuristic", "agc_code_build", "agc_codes_bytes", "agc_decode",
     "agc_decode_two_track", "agc_decode_update_static", "agc_decode_residuals", "agc_two_track_vector", "AGC_ERR_LIMIT",
-    "agc_combine_norm_sums", "agc_encode_norm_sums", "agc_encode_quantize", "agc_encode_quantize_rows", "agc_encode_quantize_with_norms", "agc_eta_balance", "agc_plan_create", "agc_plan_destroy", "agc_plan_set_first_block", "agc_plan_uses_tma",
+    "agc_combine_norm_sums", "agc_encode_norm_sums", "agc_encode_quantize", "agc_encode_quantize_rows", "agc_encode_quantize_with_norms", "agc_eta_balance", "agc_plan_create", "agc_plan_destroy", "agc_plan_encode_layout", "agc_plan_set_first_block", "agc_plan_uses_tma",
     "agc_round_host", "agc_scales_bytes", "agc_selftest_division", "agc_selftest_sqrt", "agc_strerror", "agc_version", "agc_worker_offset",
     "library_path")
 

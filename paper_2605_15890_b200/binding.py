@@ -66,6 +66,8 @@ def _load():
     L.agc_encode_quantize.restype = C.c_int
     L.agc_encode_quantize_rows.argtypes = [vp, vp, C.c_uint64, vp, vp, vp, vp]
     L.agc_encode_quantize_rows.restype = C.c_int
+    L.agc_plan_encode_layout.argtypes = [vp, i32p]
+    L.agc_plan_encode_layout.restype = C.c_int
     L.agc_encode_norm_sums.argtypes = [vp, vp, C.c_int64, vp, vp]
     L.agc_encode_norm_sums.restype = C.c_int
     L.agc_combine_norm_sums.argtypes = [C.c_int, C.c_int, f32p, f32p]
@@ -200,6 +202,13 @@ def agc_encode_quantize_rows(plan, G_rows_dev, rnd, codes_dev, scales_dev, statu
     """G_rows_dev: device array of k row addresses (a torch int64 CUDA tensor)."""
     _check(_lib.agc_encode_quantize_rows(plan, _dev(G_rows_dev), rnd, _dev(codes_dev), _dev(scales_dev),
                                          _dev(status_dev), _stream(stream)))
+
+
+def agc_plan_encode_layout(plan):
+    """dict(staged, groups, rows_staged, stages) of the plan's encoder tiling."""
+    out = np.zeros(4, np.int32)
+    _check(_lib.agc_plan_encode_layout(plan, _hp(out, C.c_int32)))
+    return {"staged": bool(out[0]), "groups": int(out[1]), "rows_staged": int(out[2]), "stages": int(out[3])}
 
 
 def agc_encode_norm_sums(plan, G_dev, ld, sumsq_dev, stream=None):

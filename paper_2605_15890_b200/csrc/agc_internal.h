@@ -137,6 +137,7 @@ struct agc_plan {
     // encode tiling
     bool use_tma = false;
     int n_groups = 0, stage_rows = 0, stages = 0, n_ops = 0;
+    int rows_staged = 0;          // partition rows brought into shared memory per pack block, all groups together
     size_t enc_smem = 0;
     // decode ring
     bool dec_ring = false;

@@ -191,6 +191,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     int max_rows = 0;
     bool stageable = build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
     pl->n_groups = int(grp_row_ptr.size()) - 1;
+    pl->rows_staged = grp_row_ptr.empty() ? 0 : int(grp_row_ptr.back());
     pl->use_tma = false;
     std::vector<AgcWorkerDesc> wdesc(n_workers);
     std::vector<AgcEntryDesc> edesc(nnz);
@@ -288,6 +289,15 @@ extern "C" int agc_plan_set_first_block(agc_plan_t *plan, int64_t first_block)
     return AGC_OK;
 }
 extern "C" int agc_plan_uses_tma(const agc_plan_t *plan) { return plan && plan->use_tma ? 1 : 0; }
+extern "C" int agc_plan_encode_layout(const agc_plan_t *plan, int32_t *out4)
+{
+    if (!plan || !out4) return AGC_ERR_ARG;
+    out4[0] = plan->use_tma ? 1 : 0;
+    out4[1] = plan->use_tma ? plan->n_groups : 0;
+    out4[2] = plan->use_tma ? plan->rows_staged : 0;
+    out4[3] = plan->use_tma ? plan->stages : 0;
+    return AGC_OK;
+}
 
 extern "C" int agc_encode_quantize(agc_plan_t *plan, const float *G_dev, int64_t ld, uint64_t round,
                                    void *codes_dev, float *scales_dev, uint32_t *status_dev, void *cuda_stream)

@@ -112,7 +112,9 @@ def partials_numpy(wl, round_index=0, d=None):
     """k x d float32 partial gradients on the host (small workloads / slices)."""
     d = wl.d if d is None else d
     r = _rng(wl.seed, 1000 + round_index)
-    if wl.value_model == "normal":
+    if wl.value_model in ("normal", "least_squares"):
+        # least_squares (cfg4): the partial gradients proper come from the harness's regression
+        # problem on the device; host-side samples of that shape are standard normal
         return r.standard_normal((wl.k, d), dtype=np.float32)
     if wl.value_model == "partition_scale":
         g = r.standard_normal((wl.k, d), dtype=np.float32)

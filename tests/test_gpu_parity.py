@@ -471,17 +471,26 @@ def test_config5_shape_one_bit_workers_and_64_realisations(agc, torch):
     assert rel <= 1e-5
 
 
-def test_config3_full_size_sampled_blocks(agc, torch):
+@pytest.mark.parametrize("builder", ["bench", "oracle"])
+def test_config3_full_size_sampled_blocks(agc, torch, builder):
     """The benchmark's own configuration (d = 25,557,032, bits from the allocator, bucket 512,
     the launch shape bench.py times): pack blocks sampled across the vector - first, last
     (ragged), segment boundaries, random ones - are recomputed one by one by the oracle from
-    the same inputs and compared bit for bit: codes, scales, decode and fused update."""
+    the same inputs and compared bit for bit: codes, scales, decode and fused update.
+    builder = bench: the very bits and weights bench.py times (the library's Algorithm 1 and
+    its solve on the cyclic support, zero coefficients dropped); oracle: bits from the
+    oracle's Algorithm 1 and the column-normalised weights (all s entries per worker)."""
     from paper_2605_15890_b200.session import Session
     wl = cfgs.config3()
     B = 512
-    bits, _ = od.bit_allocate_low_complexity(wl.p, wl.z_tot, B, b_max=8)
-    bits = np.asarray(bits, np.uint8)
-    rp, ci, a, w = _codes.cyclic_code(wl.p, bits, wl.k, wl.s, B)
+    if builder == "bench":
+        import bench
+        (rp, ci, a, w), bits = bench.build_code(agc, wl, B, "cyclic")
+        assert len(ci) < wl.n * wl.s           # the solve drove some coefficients to zero
+    else:
+        bits, _ = od.bit_allocate_low_complexity(wl.p, wl.z_tot, B, b_max=8)
+        bits = np.asarray(bits, np.uint8)
+        rp, ci, a, w = _codes.cyclic_code(wl.p, bits, wl.k, wl.s, B)
     ses = Session(wl.n, wl.k, wl.d, rp, ci, a, w, wl.p, bits, bucket=B, seed=wl.seed)
     assert ses.uses_tma
     ld = (wl.d + 3) // 4 * 4
