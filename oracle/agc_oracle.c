@@ -38,8 +38,8 @@
 #define AGC_ORACLE_STATUS_RANGE 2u      /* a code left [0, 2L]: must never happen  */
 
 /* ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers:
- * as easy as 1, 2, 3", SC'11). The paper asks only for "lightweight shared
- * random seeds" (Sec. II-B); a counter-based generator makes every draw a pure
+ * as easy as 1, 2, 3", SC'11). The paper asks only that the rounding's randomness come from cheap
+ * seeds shared by the parties (Sec. II-B); a counter-based generator makes every draw a pure
  * function of (seed, round, worker, stream position). ---- */
 void agc_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
 {
