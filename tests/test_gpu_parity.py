@@ -321,6 +321,33 @@ def test_workers_without_entries_send_the_zero_vector(agc, torch, B, direct):
     assert (ref["scales"][[1, 3, 6]] == 0).all()
 
 
+@pytest.mark.parametrize("B", [128, 512])
+def test_decode_coefficients_across_the_exponent_range(agc, torch, B):
+    """Decoding coefficients w_i S / L from the subnormal range up to 1e30: the decoder scales a
+    coefficient by a power of two where the code sits in its word, which is exact only inside
+    the normal range; smaller coefficients must take its general path and give the same bits
+    as the oracle's plain fma chain."""
+    rng = np.random.default_rng(17 + B)
+    n = k = 8
+    d = 5 * 512 + 33
+    bits = np.array([2, 3, 4, 5, 6, 7, 8, 2], np.uint8)
+    p = np.full(n, 0.1)
+    rp, ci, a, _ = _codes.cyclic_code(p, bits, k, 2, B)
+    G = rng.standard_normal((k, d)).astype(np.float32)
+    for w in ([1e-30, 1e-33, 1e-36, 1e-38, 1e-41, 1e-44, 1.0, 1e-35], [1e30, 1.0, 1e-20, 3e-34, 0.0, -1e-37, -2.5, 1e-39]):
+        w = np.array(w, np.float32)
+        out, ref = run_both(agc, torch, G, (rp, ci, a, w), p, bits, B, 3, 1, np.ones((1, n)),
+                            flags=agc.AGC_FLAG_NO_UNBIASED_CHECK)
+        assert_exact(out, ref)
+    # tiny values as well: scales near 2^-60 with ordinary weights
+    out, ref = run_both(agc, torch, G * np.float32(1e-19), (rp, ci, a, np.ones(n, np.float32)), p, bits, B, 3, 1,
+                        np.ones((1, n)), flags=agc.AGC_FLAG_NO_UNBIASED_CHECK)
+    assert_exact(out, ref)
+    out, ref = run_both(agc, torch, G * np.float32(1e-19), (rp, ci, a, np.full(n, 1e-15, np.float32)), p, bits, B, 3, 1,
+                        np.ones((1, n)), flags=agc.AGC_FLAG_NO_UNBIASED_CHECK)
+    assert_exact(out, ref)
+
+
 def test_same_round_same_bits_other_round_other_bits(agc, torch):
     wl = cfgs.config1()
     code = _codes.cyclic_code(wl.p, wl.bits, wl.k, wl.s, 512)
