@@ -57,6 +57,8 @@ extern "C" {
 #define AGC_FLAG_ALLOW_1BIT 1u         /* accept b_i = 1 (two-point quantiser; outside the paper)  */
 #define AGC_FLAG_NO_UNBIASED_CHECK 2u  /* skip the check of the unbiasedness condition             */
 #define AGC_FLAG_FORCE_DIRECT 4u       /* always use the direct-load encode kernel (no TMA staging) */
+#define AGC_FLAG_NO_ROW_DECODE 8u      /* vectors of fewer pack blocks than SMs decode with the staged kernel as
+                                          well, not with the warp-per-row kernel for short vectors */
 
 /* bits OR-ed into *status_dev by the kernels */
 #define AGC_STATUS_NONFINITE 1u  /* a bucket had a NaN/Inf sum of squares: sent as zeros, scale 0 */

@@ -10,7 +10,7 @@ The binding is loaded on first attribute access, so that `paper_2605_15890_b200.
 import importlib
 
 _BINDING_NAMES = (
-    "AGC_CODE_INTERVAL", "AGC_CODE_SUPPORT", "AGC_FLAG_ALLOW_1BIT", "AGC_FLAG_FORCE_DIRECT",
+    "AGC_CODE_INTERVAL", "AGC_CODE_SUPPORT", "AGC_FLAG_ALLOW_1BIT", "AGC_FLAG_FORCE_DIRECT", "AGC_FLAG_NO_ROW_DECODE",
     "AGC_FLAG_NO_UNBIASED_CHECK", "AGC_STATUS_NONFINITE", "AGC_STATUS_TIMEOUT", "AgcError",
     "AGC_ALLOC_GREEDY", "AGC_ALLOC_RELAXATION", "agc_allocation_upper_bound", "agc_bit_allocate", "agc_bit_allocate_dp", "agc_bit_allocate_heuristic", "agc_code_build", "agc_codes_bytes", "agc_decode",
     "agc_decode_two_track", "agc_decode_update_static", "agc_decode_residuals", "agc_two_track_vector", "AGC_ERR_LIMIT",

@@ -15,6 +15,7 @@ _LIB_PATH = os.path.join(_HERE, "libagc.so")
 AGC_FLAG_ALLOW_1BIT = 1
 AGC_FLAG_NO_UNBIASED_CHECK = 2
 AGC_FLAG_FORCE_DIRECT = 4
+AGC_FLAG_NO_ROW_DECODE = 8
 AGC_STATUS_NONFINITE = 1
 AGC_STATUS_TIMEOUT = 4
 AGC_CODE_INTERVAL = 0

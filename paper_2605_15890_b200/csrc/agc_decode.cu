@@ -206,6 +206,169 @@ __global__ void __launch_bounds__(256) agc_decode_kernel(const AgcDecParams P)
     }
 }
 
+// ------------------------------------------------------------------ short vectors
+// A vector of fewer pack blocks than SMs leaves most of the GPU idle when one warp owns a
+// whole block, and the chain of fmas over the workers (one after the other, the defining
+// order) is then the whole run time. Here a CTA of four warps owns a block and each warp one
+// ROW of it, the 128 coordinates 128c + 4*lane + e of row c: a quarter of the unpacking each.
+// The four codes of a lane's row are 4 * b consecutive bits of its 16-code slice; they are
+// fetched with at most two word loads and one funnel shift, for every width alike. The
+// workers that contribute are listed in shared memory first (coefficient of each row, address
+// of the block's words, width), in ascending order, so that the loop over them depends on no
+// global load but the words', which are fetched eight workers ahead.
+struct __align__(16) AgcRowWorker {
+    float cs[4];                 // coefficient w_i S / L_i of each row of the block (0 .. 3)
+    const uint32_t *words;       // the worker's words of this pack block
+    uint32_t bits;               // 0: the worker does not contribute
+    uint32_t pad;
+};
+#define AGC_ROWS_AHEAD 8
+
+template <int BITS>
+__device__ __forceinline__ void row_levels_fma(uint32_t x, float cstep, float (&acc)[4])
+{
+    constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const uint32_t code = (x >> (e * BITS)) & MASK;
+        float level;
+        if constexpr (BITS >= 2) level = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f + (float)L);   // code - L, exact
+        else level = __uint_as_float(0xBF000000u ^ (code << 31));                                               // code - 0.5
+        acc[e] = __fmaf_rn(cstep, level, acc[e]);
+    }
+}
+
+__device__ __forceinline__ void load4(const float *base, long long m, long long d, bool vec, float (&v)[4])
+{
+    if (vec && m + 3 < d) {
+        const float4 x = *reinterpret_cast<const float4 *>(base + m);
+        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = (m + e < d) ? base[m + e] : 0.0f;
+    }
+}
+__device__ __forceinline__ void store4(float *base, long long m, long long d, bool vec, const float (&v)[4])
+{
+    if (vec && m + 3 < d) {
+        *reinterpret_cast<float4 *>(base + m) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (m + e < d) base[m + e] = v[e];
+    }
+}
+
+// One CTA per pack block, one warp per row of 128 coordinates; one realisation (g_hat and /
+// or the fused update) or the collapsed multi-realisation update. Same arithmetic per
+// coordinate as the other decoders. Dynamic shared memory: 2 n records + 16 bytes.
+template <int RB, bool COLLAPSED>
+__global__ void __launch_bounds__(128) agc_decode_rows_kernel(const AgcDecParams P)
+{
+    extern __shared__ __align__(16) unsigned char rows_smem[];
+    AgcRowWorker *s_raw = reinterpret_cast<AgcRowWorker *>(rows_smem);
+    AgcRowWorker *s_list = s_raw + P.n;
+    int *s_count = reinterpret_cast<int *>(s_list + P.n);
+    const int lane = threadIdx.x & 31, c = threadIdx.x >> 5;
+    const long long q = blockIdx.x;
+    // every worker's record for this block, by all threads
+    for (int i = threadIdx.x; i < P.n; i += blockDim.x) {
+        AgcRowWorker rec;
+        float wgt = 0.0f;
+        bool used;
+        if (COLLAPSED) {
+            const float we = P.weff[i];
+            used = we != 0.0f;
+            if (used) wgt = __fmul_rn(P.w[i], we);
+        } else {
+            used = P.masks[i] != 0;
+            if (used) wgt = P.w[i];
+        }
+        const uint32_t bits = P.bits[i];
+        rec.bits = used ? bits : 0u;
+        rec.pad = 0u;
+        rec.words = P.codes + P.word_off[i] + q * 16 * (long long)bits;
+        const float dstep = bits >= 2 ? (float)(1.0 / (double)((1 << (bits - 1)) - 1)) : 2.0f;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const long long beta = (q * (4 / RB) + r / RB) >> P.scale_shift;
+            const float S = (used && beta < P.nb) ? __ldg(P.scales + (long long)i * P.nb + beta) : 0.0f;
+            rec.cs[r] = __fmul_rn(__fmul_rn(wgt, S), dstep);
+        }
+        s_raw[i] = rec;
+    }
+    __syncthreads();
+    if (c == 0) {
+        // ascending list of the workers that contribute
+        int cnt = 0;
+        for (int base = 0; base < P.n; base += 32) {
+            const int i = base + lane;
+            const bool used = i < P.n && s_raw[i].bits != 0u;
+            const unsigned vote = __ballot_sync(0xffffffffu, used);
+            if (used) s_list[cnt + __popc(vote & ((1u << lane) - 1u))] = s_raw[i];
+            cnt += __popc(vote);
+        }
+        if (lane == 0) *s_count = cnt;
+    }
+    __syncthreads();
+    const int cnt = *s_count;
+    const long long m = q * AGC_BLOCK + c * 128 + 4 * lane;
+    if (m >= P.d) return;
+    const bool vec = (P.d & 3) == 0;
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int base = 0; base < cnt; base += AGC_ROWS_AHEAD) {
+        float cs[AGC_ROWS_AHEAD];
+        uint32_t bits[AGC_ROWS_AHEAD], lo[AGC_ROWS_AHEAD], hi[AGC_ROWS_AHEAD], sh[AGC_ROWS_AHEAD];
+#pragma unroll
+        for (int k = 0; k < AGC_ROWS_AHEAD; ++k) {
+            bits[k] = 0u;
+            if (base + k < cnt) {
+                const AgcRowWorker &rec = s_list[base + k];
+                bits[k] = rec.bits;
+                cs[k] = rec.cs[c];
+                const uint32_t start = ((uint32_t)lane * 16u + 4u * (uint32_t)c) * bits[k];   // bit offset of the row's four codes
+                sh[k] = start & 31u;
+                lo[k] = __ldg(rec.words + (start >> 5));
+                // the four codes end inside the block (the last ones exactly at its end): a
+                // second word is read only where it exists
+                hi[k] = (sh[k] + 4u * bits[k] > 32u) ? __ldg(rec.words + (start >> 5) + 1) : 0u;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < AGC_ROWS_AHEAD; ++k) {
+            const uint32_t x = __funnelshift_r(lo[k], hi[k], sh[k]);
+            switch (bits[k]) {
+                case 0: break;
+                case 1: row_levels_fma<1>(x, cs[k], acc); break;
+                case 2: row_levels_fma<2>(x, cs[k], acc); break;
+                case 3: row_levels_fma<3>(x, cs[k], acc); break;
+                case 4: row_levels_fma<4>(x, cs[k], acc); break;
+                case 5: row_levels_fma<5>(x, cs[k], acc); break;
+                case 6: row_levels_fma<6>(x, cs[k], acc); break;
+                case 7: row_levels_fma<7>(x, cs[k], acc); break;
+                default: row_levels_fma<8>(x, cs[k], acc); break;
+            }
+        }
+    }
+    if (COLLAPSED) {
+        float b[4];
+        load4(P.beta, m, P.d, vec, b);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) b[e] = __fsub_rn(b[e], acc[e]);
+        store4(P.beta, m, P.d, vec, b);
+    } else {
+        if (P.ghat) store4(P.ghat, m, P.d, vec, acc);
+        if (P.beta) {
+            float b[4];
+            load4(P.beta, m, P.d, vec, b);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) b[e] = __fmaf_rn(-P.lr0, acc[e], b[e]);
+            store4(P.beta, m, P.d, vec, b);
+        }
+    }
+}
+
 // weff_i = sum_r lr_r * I_{r,i}, summed in order of r
 __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *lr, int n, int R, float *weff)
 {
@@ -969,6 +1132,18 @@ int launch_multi_rb(const AgcDecParams &P, int sm_count, int smem_optin, cudaStr
     return AGC_OK;
 }
 
+size_t rows_smem_bytes(int n) { return 2 * sizeof(AgcRowWorker) * size_t(n) + 16; }
+
+template <bool COLLAPSED>
+void launch_rows(const AgcDecParams &P, cudaStream_t stream)
+{
+    const int grid = (int)P.nblk;   // one CTA of four warps per pack block
+    const size_t smem = rows_smem_bytes(P.n);
+    if (P.rows_per_bucket == 4) agc_decode_rows_kernel<4, COLLAPSED><<<grid, 128, smem, stream>>>(P);
+    else if (P.rows_per_bucket == 2) agc_decode_rows_kernel<2, COLLAPSED><<<grid, 128, smem, stream>>>(P);
+    else agc_decode_rows_kernel<1, COLLAPSED><<<grid, 128, smem, stream>>>(P);
+}
+
 template <bool COLLAPSED>
 void launch(const AgcDecParams &P, int grid, cudaStream_t stream)
 {
@@ -1024,6 +1199,22 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
         // the R updates in order, from the rows just written
         const long long want = (plan->d + 255) / 256, cap = (long long)plan->sm_count * 8;
         agc_apply_updates_kernel<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(ghat, plan->d_lr, R, plan->d, beta);
+        return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
+    }
+    if (plan->dec_ring && plan->nblk <= plan->sm_count && !(plan->flags & AGC_FLAG_NO_ROW_DECODE)) {
+        // fewer pack blocks than SMs: a warp per row of a block, plain loads (the messages of such
+        // a vector are a few hundred KB at most)
+        if (collapsed) {
+            launch_rows<true>(P, stream);
+        } else {
+            // one launch per realisation, in order: realisation r sees beta after r - 1
+            for (int r = 0; r < R; ++r) {
+                P.masks = masks + (size_t)r * plan->n;
+                P.ghat = ghat ? ghat + (size_t)r * plan->d : nullptr;
+                P.lr0 = (beta && lr_host) ? lr_host[r] : 0.0f;
+                launch_rows<false>(P, stream);
+            }
+        }
         return cudaGetLastError() == cudaSuccess ? AGC_OK : AGC_ERR_CUDA;
     }
     if (plan->dec_ring) {
@@ -1100,6 +1291,13 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
         cudaFuncSetAttribute(agc_decode_multi_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
         cudaFuncSetAttribute(agc_decode_multi_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
         cudaFuncSetAttribute(agc_decode_multi_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
+        return AGC_ERR_CUDA;
+    if (cudaFuncSetAttribute(agc_decode_rows_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_rows_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_rows_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_rows_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_rows_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
+        cudaFuncSetAttribute(agc_decode_rows_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
         return AGC_ERR_CUDA;
     plan->smem_optin = smem_optin;
     plan->dec_ring = true;

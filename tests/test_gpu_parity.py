@@ -102,7 +102,7 @@ def test_config1_all_rounds_bit_exact(agc, torch):
 
 @pytest.mark.parametrize("d", [1, 3, 127, 128, 129, 511, 512, 513, 1000, 4097, 70001])
 @pytest.mark.parametrize("B", [128, 256, 512])
-@pytest.mark.parametrize("direct", [False, True])
+@pytest.mark.parametrize("direct", [False, True, "ring"])
 def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
     rng = np.random.default_rng(d * 7 + B)
     n = k = 8
@@ -111,10 +111,15 @@ def test_ragged_sizes_all_bit_widths(agc, torch, d, B, direct):
     code = _codes.cyclic_code(p, bits, k, 3, B)
     G = (rng.standard_normal((k, d)) * 10.0 ** rng.uniform(-3, 2, (k, 1))).astype(np.float32)
     masks = (rng.random((2, n)) > 0.3).astype(np.uint8)
-    out, ref = run_both(agc, torch, G, code, p, bits, B, 1234 + d, 5, masks,
-                        flags=agc.AGC_FLAG_FORCE_DIRECT if direct else 0, ld_pad=4 if d % 2 else 0)
+    # three routes: staged encoder + the short-vector decoder (these lengths are below one pack
+    # block per SM), both direct-load kernels, staged encoder + staged (ring) decoder
+    flags = agc.AGC_FLAG_FORCE_DIRECT if direct is True else agc.AGC_FLAG_NO_ROW_DECODE if direct == "ring" else 0
+    out, ref = run_both(agc, torch, G, code, p, bits, B, 1234 + d, 5, masks, flags=flags, ld_pad=4 if d % 2 else 0,
+                        beta0=rng.standard_normal(d).astype(np.float32), lr=np.array([0.01, 0.02], np.float32))
     assert_exact(out, ref)
-    assert out["tma"] == (not direct)
+    assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
+    assert np.abs(out["beta_fused"] - ref["beta"]).max() <= 1e-5 * np.abs(ref["beta"]).max()
+    assert out["tma"] == (direct is not True)
 
 
 @pytest.mark.parametrize("kind", ["identity", "interval", "s1", "s_eq_k", "wide_rows", "many_groups", "many_workers", "scattered", "thousands"])
@@ -216,8 +221,10 @@ def test_seeded_random_shapes_codes_and_masks(agc, torch, case):
     beta0 = rng.standard_normal(d).astype(np.float32)
     seed = int(rng.integers(0, 2**63)) * 2 + 1
     rnd = int(rng.integers(0, 2**63))
+    # short vectors: every other case keeps the staged decoder instead of the warp-per-row kernel
+    flags = agc.AGC_FLAG_NO_ROW_DECODE if case % 2 else 0
     out, ref = run_both(agc, torch, G, code, p, bits, B, seed, rnd, masks, lr=lr, beta0=beta0,
-                        ld_pad=int(rng.choice([0, 4, 36])))
+                        ld_pad=int(rng.choice([0, 4, 36])), flags=flags)
     assert_exact(out, ref)
     assert (out["beta_seq"].view(np.uint32) == ref["beta"].view(np.uint32)).all()
     scale = max(np.abs(ref["beta"]).max(), 1e-30)
