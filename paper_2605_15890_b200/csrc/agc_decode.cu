@@ -383,6 +383,12 @@ __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *
 #ifndef AGC_DEC_PREFETCH
 #define AGC_DEC_PREFETCH 1
 #endif
+#ifndef AGC_DEC_LUT2
+#define AGC_DEC_LUT2 1
+#endif
+// static shared memory of the ring kernel: the table of 2-bit level pairs (128 bytes), padded
+// to the 1 KiB alignment of the dynamic part
+#define AGC_DEC_STATIC_SMEM 1024
 // ------------------------------------------------------------------ ring kernel
 // Persistent CTAs. A tile is AGC_DEC_QT consecutive pack blocks of one group of received
 // workers: the producer warp brings each worker's chunk (its words of those blocks are
@@ -435,7 +441,7 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 template <int BITS, bool TWO = false>
 __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uint32_t to, int lane,
                                                 const float (&ws_row)[4], float (&acc)[16],
-                                                const float (&ws2_row)[4], float (&acc2)[16])
+                                                const float (&ws2_row)[4], float (&acc2)[16], uint32_t lut2)
 {
     constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
     constexpr uint32_t MASK = (1u << BITS) - 1u;
@@ -471,6 +477,31 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
         for (int t = 0; t <= H; ++t) W[t] = lds32(src + 4 * t);
         odd_width_slice<BITS>(W, lane, lw);
     }
+#if AGC_DEC_LUT2
+    // 2-bit codes, two at a time: a nibble of the word indexes a table of 16 level pairs
+    // (code0 - 1, code1 - 1) in shared memory. The table is 128 bytes, one per bank pair, so
+    // any 32 lanes read it without a bank conflict; the pair feeds the packed fma directly:
+    // shift + logic operation + shared load per two codes, no subtraction.
+    if constexpr (BITS == 2) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t off = (j == 0 ? A[0] << 3 : A[0] >> (4 * j - 3)) & 0x78u;   // 8 * nibble j
+            float2 level;
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(level.x), "=f"(level.y) : "r"(lut2 + off));
+            const float c = cstep_row[j >> 1];
+            const float2 r = __ffma2_rn(make_float2(c, c), level, make_float2(acc[2 * j], acc[2 * j + 1]));
+            acc[2 * j] = r.x;
+            acc[2 * j + 1] = r.y;
+            if constexpr (TWO) {
+                const float c2 = cstep2_row[j >> 1];
+                const float2 r2 = __ffma2_rn(make_float2(c2, c2), level, make_float2(acc2[2 * j], acc2[2 * j + 1]));
+                acc2[2 * j] = r2.x;
+                acc2[2 * j + 1] = r2.y;
+            }
+        }
+        return;
+    }
+#endif
     // two coordinates at a time: the subtraction and the fma are packed instructions (two
     // independent IEEE fp32 operations each), which halves their issue slots
 #pragma unroll
@@ -585,6 +616,10 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     uint8_t *s_raw_allb = s_raw_b + P.n;
     float *s_w2 = reinterpret_cast<float *>(smem + P.w2_offset);   // second decoder of the received workers
 
+    // level pairs of two 2-bit codes: entry v = (v & 3) - 1, (v >> 2) - 1
+    __shared__ __align__(128) float2 s_lut2[16];
+    const uint32_t lut2 = smem_addr(s_lut2);
+    if (threadIdx.x < 16) s_lut2[threadIdx.x] = make_float2((float)(threadIdx.x & 3) - 1.0f, (float)(threadIdx.x >> 2) - 1.0f);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -773,7 +808,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                 ws2_row[bk * RB + cc] = ws2;                                                    \
             }                                                                                   \
         }                                                                                       \
-        ring_add_worker<B, TWO>(chunk, tl, to, lane, ws_row, acc, ws2_row, acc2);               \
+        ring_add_worker<B, TWO>(chunk, tl, to, lane, ws_row, acc, ws2_row, acc2, lut2);         \
     }
                         switch (bits) {
                             case 1: AGC_DEC_RUN(1) break;
@@ -1086,8 +1121,9 @@ int ring_layout(int n, int smem_optin, size_t *smem_out, uint32_t *w2_offset)
     tail = (tail + 15) & ~size_t(15);
     const size_t w2_rel = tail;
     tail += sizeof(float) * size_t(n) + 16;
-    if (size_t(smem_optin) < tail + 2 * stage_bytes) return 0;
-    long long stages = (long long)((size_t(smem_optin) - tail) / stage_bytes);
+    const size_t budget = size_t(smem_optin) - AGC_DEC_STATIC_SMEM;   // the kernel's static shared memory is set aside
+    if (budget < tail + 2 * stage_bytes) return 0;
+    long long stages = (long long)((budget - tail) / stage_bytes);
     if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
     *smem_out = size_t(stages) * stage_bytes + tail;
     *w2_offset = uint32_t(size_t(stages) * stage_bytes + w2_rel);
@@ -1282,8 +1318,9 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
     plan->dec2_stages = ring_layout<AGC_DEC_QT2>(plan->n, smem_optin, &plan->dec2_smem, &plan->dec2_w2_offset);
     if (plan->dec_stages < 2 || plan->dec2_stages < 2) return AGC_OK;
     // the limit is an attribute of the kernel, shared by all plans: the device's opt-in maximum
-    if (!ring_set_smem<0, AGC_DEC_QT>(smem_optin) || !ring_set_smem<1, AGC_DEC_QT>(smem_optin) ||
-        !ring_set_smem<2, AGC_DEC_QT2>(smem_optin))
+    const int ring_dyn = smem_optin - AGC_DEC_STATIC_SMEM;
+    if (!ring_set_smem<0, AGC_DEC_QT>(ring_dyn) || !ring_set_smem<1, AGC_DEC_QT>(ring_dyn) ||
+        !ring_set_smem<2, AGC_DEC_QT2>(ring_dyn))
         return AGC_ERR_CUDA;
     if (cudaFuncSetAttribute(agc_decode_multi_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
         cudaFuncSetAttribute(agc_decode_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess ||
