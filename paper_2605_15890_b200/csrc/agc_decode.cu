@@ -504,6 +504,7 @@ __device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uin
 #endif
     // two coordinates at a time: the subtraction and the fma are packed instructions (two
     // independent IEEE fp32 operations each), which halves their issue slots
+    if constexpr (!(AGC_DEC_LUT2 && BITS == 2))
 #pragma unroll
     for (int t = 0; t < 16; t += 2) {
         float lv[2];
