@@ -16,7 +16,7 @@
 #endif
 #define AGC_ENC_TABLE_BYTES_MAX (48 * 1024)  // shared-memory budget of the staged encoder's tables
 #ifndef AGC_PRODUCER_SLEEP_NS
-#define AGC_PRODUCER_SLEEP_NS 32u  // cap of the producer warps' sleep between tries of a wait
+#define AGC_PRODUCER_SLEEP_NS 256u  // cap of the producer warps' sleep between tries of a wait
 #endif
 #define AGC_MAX_R 4096         // straggler realisations per decode call
 #ifndef AGC_DEC_QT

@@ -34,9 +34,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // Bounded wait. A warp that finds the phase incomplete sleeps between tries (32 ns doubling
 // up to MAX_SLEEP_NS) instead of spinning, so that it does not take issue slots from the
 // warps still working; a producer warp, whose wake-up delay adds to the refill latency of a
-// ring stage, uses a short cap. After 2^22 tries (a quarter of a second at the least with
-// the hardware's own suspension of each try) it gives up, records it and lets the caller
-// unwind.
+// ring stage, uses a shorter cap. After 2^22 tries (about a second with a cap of 256 ns,
+// two with 512 ns) it gives up, records it and lets the caller unwind.
 template <uint32_t MAX_SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait_loop(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
