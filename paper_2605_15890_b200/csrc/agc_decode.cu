@@ -400,9 +400,10 @@ struct __align__(16) AgcDecWorker {
     long long word_off;    // word offset of the worker's message
     long long scales_off;  // i * nb
     float weight;          // w_i, or w_i * (sum_r lr_r I_ri) in the collapsed mode
+    float dstep;           // 1 / L_i as fp32 (2 for one-bit codes): distance between two levels
     uint32_t soff;         // byte offset of the worker's chunk inside a stage
-    uint32_t bits;
-    uint32_t run;          // at the first worker of a run of equal widths inside a group: its length
+    uint16_t bits;
+    uint16_t run;          // at the first worker of a run of equal widths inside a group: its length
 };
 
 // (a & b) | c in one logic instruction
@@ -432,49 +433,53 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     return v;
 }
 
-// One worker's contribution to the lane's 16 accumulators, read from the staged chunk
-// (chunk: its 32-bit shared-memory address).
-//   tl   warp * 64 + lane * 2 (even widths: byte offset of the lane's slice is tl * BITS)
-//   to   warp * 64 + (lane / 2) * 4 (odd widths: a pair of lanes shares BITS words)
+// One worker's contribution to the lane's 16 accumulators, read from the staged chunk.
+//   src    32-bit shared-memory address of the lane's words of the worker's block: the chunk
+//          plus ring_lane_offset<BITS>()
+//   cstep  per 128-coordinate row, (w_i * scale) * (1 / L_i): the step of one level
 // The integer code c becomes the float 2^23 + c by OR-ing it into the mantissa of 2^23
 // (one byte permute for 8-bit codes); level = that - (2^23 + L) is exact.
+//   tl   warp * 64 + lane * 2 (even widths: byte offset of the lane's slice is tl * BITS)
+//   to   warp * 64 + (lane / 2) * 4 (odd widths: a pair of lanes shares BITS words)
+template <int BITS>
+__device__ __forceinline__ uint32_t ring_lane_offset(uint32_t tl, uint32_t to, int lane)
+{
+    if constexpr (BITS % 2 == 0) return tl * BITS;
+    else return to * BITS + ((lane & 1) ? 4u * ((BITS - 1) / 2) : 0u);
+}
+
+// The lane's words of one worker's block, as they lie in the staged chunk.
+template <int BITS>
+__device__ __forceinline__ void ring_load_words(uint32_t src, uint32_t (&W)[LaneWords<BITS>::NACC])
+{
+    constexpr int NW = LaneWords<BITS>::NACC;
+    if constexpr (BITS % 2 == 0 && NW == 4) {
+        const uint4 v = lds128(src);
+        W[0] = v.x; W[1] = v.y; W[2] = v.z; W[3] = v.w;
+    } else if constexpr (BITS % 2 == 0 && NW == 2) {
+        const uint2 v = lds64(src);
+        W[0] = v.x; W[1] = v.y;
+    } else {
+#pragma unroll
+        for (int t = 0; t < NW; ++t) W[t] = lds32(src + 4 * t);
+    }
+}
+
 template <int BITS, bool TWO = false>
-__device__ __forceinline__ void ring_add_worker(uint32_t chunk, uint32_t tl, uint32_t to, int lane,
-                                                const float (&ws_row)[4], float (&acc)[16],
-                                                const float (&ws2_row)[4], float (&acc2)[16], uint32_t lut2)
+__device__ __forceinline__ void ring_add_worker(const uint32_t (&W)[LaneWords<BITS>::NACC], int lane,
+                                                const float (&cstep_row)[4], float (&acc)[16],
+                                                const float (&cstep2_row)[4], float (&acc2)[16], uint32_t lut2)
 {
     constexpr uint32_t L = BITS >= 2 ? (1u << (BITS >= 2 ? BITS - 1 : 1)) - 1u : 0u;
     constexpr uint32_t MASK = (1u << BITS) - 1u;
-    constexpr float DSTEP = BITS >= 2 ? (float)(1.0 / (double)(BITS >= 2 ? L : 1u)) : 2.0f;
     constexpr int NACC = LaneWords<BITS>::NACC;
-    float cstep_row[4], cstep2_row[4];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        cstep_row[c] = __fmul_rn(ws_row[c], DSTEP);
-        cstep2_row[c] = TWO ? __fmul_rn(ws2_row[c], DSTEP) : 0.0f;
-    }
     LaneWords<BITS> lw;
     uint32_t (&A)[NACC + 1] = lw.A;
     A[NACC] = 0u;
     if constexpr (BITS % 2 == 0) {
-        constexpr int NW = BITS / 2;
-        const uint32_t src = chunk + tl * BITS;
-        if constexpr (NW == 4) {
-            const uint4 v = lds128(src);
-            A[0] = v.x; A[1] = v.y; A[2] = v.z; A[3] = v.w;
-        } else if constexpr (NW == 2) {
-            const uint2 v = lds64(src);
-            A[0] = v.x; A[1] = v.y;
-        } else {
 #pragma unroll
-            for (int t = 0; t < NW; ++t) A[t] = lds32(src + 4 * t);
-        }
+        for (int t = 0; t < NACC; ++t) A[t] = W[t];
     } else {
-        constexpr int H = (BITS - 1) / 2;
-        const uint32_t src = chunk + to * BITS + ((lane & 1) ? 4 * H : 0);
-        uint32_t W[H + 1];
-#pragma unroll
-        for (int t = 0; t <= H; ++t) W[t] = lds32(src + 4 * t);
         odd_width_slice<BITS>(W, lane, lw);
     }
 #if AGC_DEC_LUT2
@@ -619,8 +624,8 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
 
     // level pairs of two 2-bit codes: entry v = (v & 3) - 1, (v >> 2) - 1
     __shared__ __align__(128) float2 s_lut2[16];
-    const uint32_t lut2 = smem_addr(s_lut2);
     if (threadIdx.x < 16) s_lut2[threadIdx.x] = make_float2((float)(threadIdx.x & 3) - 1.0f, (float)(threadIdx.x >> 2) - 1.0f);
+    const uint32_t lut2 = smem_addr(s_lut2);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -676,8 +681,9 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
             wk.word_off = my_off;
             wk.scales_off = (long long)i * P.nb;
             wk.weight = s_raw_w[i];
+            wk.dstep = b >= 2 ? (float)(1.0 / (double)((1u << (b - 1)) - 1u)) : 2.0f;
             wk.soff = soff;
-            wk.bits = b;
+            wk.bits = (uint16_t)b;
             wk.run = 1;
             if (TWO) s_w2[nrecv] = P.v[i];
             s_wk[nrecv++] = wk;
@@ -786,30 +792,47 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                 else fetch_scales(T + gridDim.x, 0, sc_next);
                 // parameters of the block: read early, used after the last group
                 if (!TWO && g == n_groups - 1 && P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
+                // the lane's worker of the group: step of one level per scale of the block,
+                // (w_i * scale) * (1 / L_i), handed to the other lanes by a shuffle
+                float cs[4 / RB], cs2[4 / RB];
+                {
+                    const bool mine = lane < nr;
+                    const float weight = mine ? s_wk[r0 + lane].weight : 0.0f;
+                    const float dstep = mine ? s_wk[r0 + lane].dstep : 0.0f;
+                    const float weight2 = TWO && mine ? s_w2[r0 + lane] : 0.0f;
+#pragma unroll
+                    for (int bk = 0; bk < 4 / RB; ++bk) {
+                        cs[bk] = __fmul_rn(__fmul_rn(weight, sc[bk]), dstep);
+                        cs2[bk] = TWO ? __fmul_rn(__fmul_rn(weight2, sc[bk]), dstep) : 0.0f;
+                    }
+                }
                 ok = mbar_wait(&full[s], parity, flags);
                 if (!ok) break;
                 if (active) {
                     const uint32_t stage = smem_addr(smem) + (uint32_t)s * stage_bytes;
-                    // runs of workers of equal width: one dispatch per run
+                    // runs of workers of equal width: one dispatch per run; the chunks of a run
+                    // follow one another in the stage
                     for (int r = 0; r < nr;) {
                         const int run = (int)s_wk[r0 + r].run;
                         const uint32_t bits = s_wk[r0 + r].bits;
+                        const uint32_t chunk0 = stage + s_wk[r0 + r].soff;
 #define AGC_DEC_RUN(B)                                                                          \
-    for (int j = 0; j < run; ++j) {                                                             \
-        const float weight = s_wk[r0 + r + j].weight;                                           \
-        const uint32_t chunk = stage + s_wk[r0 + r + j].soff;                                   \
-        const float weight2 = TWO ? s_w2[r0 + r + j] : 0.0f;                                    \
-        float ws_row[4], ws2_row[4];                                                            \
-        _Pragma("unroll") for (int bk = 0; bk < 4 / RB; ++bk) {                                 \
-            const float S = __shfl_sync(0xffffffffu, sc[bk], r + j);                            \
-            const float ws = __fmul_rn(weight, S);                                              \
-            const float ws2 = TWO ? __fmul_rn(weight2, S) : 0.0f;                               \
-            _Pragma("unroll") for (int cc = 0; cc < RB; ++cc) {                                 \
-                ws_row[bk * RB + cc] = ws;                                                      \
-                ws2_row[bk * RB + cc] = ws2;                                                    \
+    {                                                                                           \
+        uint32_t src = chunk0 + ring_lane_offset<B>(tl, to, lane);                              \
+        for (int j = r; j < r + run; ++j, src += qt * 64u * B) {                                \
+            uint32_t W[LaneWords<B>::NACC];                                                     \
+            float cstep_row[4], cstep2_row[4];                                                  \
+            ring_load_words<B>(src, W);                                                         \
+            _Pragma("unroll") for (int bk = 0; bk < 4 / RB; ++bk) {                             \
+                const float c = __shfl_sync(0xffffffffu, cs[bk], j);                            \
+                const float c2 = TWO ? __shfl_sync(0xffffffffu, cs2[bk], j) : 0.0f;             \
+                _Pragma("unroll") for (int cc = 0; cc < RB; ++cc) {                             \
+                    cstep_row[bk * RB + cc] = c;                                                \
+                    cstep2_row[bk * RB + cc] = c2;                                              \
+                }                                                                               \
             }                                                                                   \
+            ring_add_worker<B, TWO>(W, lane, cstep_row, acc, cstep2_row, acc2, lut2);           \
         }                                                                                       \
-        ring_add_worker<B, TWO>(chunk, tl, to, lane, ws_row, acc, ws2_row, acc2, lut2);         \
     }
                         switch (bits) {
                             case 1: AGC_DEC_RUN(1) break;
