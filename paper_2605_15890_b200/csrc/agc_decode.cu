@@ -490,9 +490,10 @@ __device__ __forceinline__ void ring_add_worker(const uint32_t (&W)[LaneWords<BI
     if constexpr (BITS == 2) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const uint32_t off = (j == 0 ? A[0] << 3 : A[0] >> (4 * j - 3)) & 0x78u;   // 8 * nibble j
+            // table address: 8 * nibble j merged into the 128-byte aligned base by one logic operation
+            const uint32_t addr = and_or(j == 0 ? A[0] << 3 : A[0] >> (4 * j - 3), 0x78u, lut2);
             float2 level;
-            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(level.x), "=f"(level.y) : "r"(lut2 + off));
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(level.x), "=f"(level.y) : "r"(addr));
             const float c = cstep_row[j >> 1];
             const float2 r = __ffma2_rn(make_float2(c, c), level, make_float2(acc[2 * j], acc[2 * j + 1]));
             acc[2 * j] = r.x;
@@ -790,8 +791,13 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                 for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = sc_next[bk];
                 if (g + 1 < n_groups) fetch_scales(T, g + 1, sc_next);
                 else fetch_scales(T + gridDim.x, 0, sc_next);
-                // parameters of the block: read early, used after the last group
-                if (!TWO && g == n_groups - 1 && P.beta && active) load16(P.beta, q, lane, P.d, vec, b);
+                // parameters of the block: asked into L2 early (one 128-byte line per lane of the
+                // first half-warp), read after the last group; holding them in registers across the
+                // group instead costs 16 registers where the unpack needs them
+                if (!TWO && g == n_groups - 1 && P.beta && active && lane < 16) {
+                    const long long m = (long long)q * AGC_BLOCK + 32 * lane;
+                    if (m < P.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.beta + m));
+                }
                 // the lane's worker of the group: step of one level per scale of the block,
                 // (w_i * scale) * (1 / L_i), handed to the other lanes by a shuffle
                 float cs[4 / RB], cs2[4 / RB];
@@ -857,7 +863,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                 if (P.ghat_v) store16(P.ghat_v, q, lane, P.d, vec, acc2);
                 if (P.beta) adam_update16(P, q, lane, vec, acc, acc2);
             } else if (ok && active) {
-                if (n_groups == 0 && P.beta) load16(P.beta, q, lane, P.d, vec, b);
+                if (P.beta) load16(P.beta, q, lane, P.d, vec, b);
                 if (COLLAPSED) {
 #pragma unroll
                     for (int t = 0; t < 16; ++t) b[t] = __fsub_rn(b[t], acc[t]);
