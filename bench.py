@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 #   dram__bytes_read.sum + dram__bytes_write.sum per launch of the encode kernel
 NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 143.80}   # captured at d = 16,777,216 (messages larger than L2)
 #   smsp__inst_executed.sum per (worker, pack block) task of the encode kernel
-NCU_WARP_INST_PER_TASK = {"cfg3": 305.1}
+NCU_WARP_INST_PER_TASK = {"cfg3": 306.5}
 
 
 def workload(name):
