@@ -607,12 +607,12 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
     constexpr bool TWO = MODE == 2;
     extern __shared__ __align__(1024) unsigned char smem[];
     const int stages = P.stages;
-    const uint32_t stage_bytes = QT * 64u * AGC_DEC_GROUP_BITS;
+    const uint32_t stage_bytes = QT * 64u * P.group_bits;
     // Tile height of this launch: QT blocks for long vectors, fewer when the vector has too
     // few blocks to give every SM a full tile. A shorter tile leaves room in a stage for a
     // wider group of workers, so that a short vector passes the ring in fewer steps.
     const uint32_t qt = (uint32_t)P.qt;
-    const uint32_t cap_bits = AGC_DEC_GROUP_BITS * QT / qt;
+    const uint32_t cap_bits = P.group_bits * QT / qt;
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)stages * stage_bytes);
     uint64_t *empty = full + AGC_DEC_MAX_STAGES;
     volatile int *flags = reinterpret_cast<volatile int *>(empty + AGC_DEC_MAX_STAGES);  // abort x2, n_groups
@@ -1141,23 +1141,36 @@ cudaError_t launch_ring(const AgcDecParams &P, int grid, size_t smem, cudaStream
 }
 
 // Shared-memory layout of the ring decoder for a tile of QT blocks: stages, then the tables.
-// Returns the ring depth (0: does not fit) and the total size / offset of the second weights.
+// Wide groups of workers cost less than many narrow ones (a wait, the scales and a dispatch
+// per group and warp), so the ring is as deep as it can be (at most AGC_DEC_MAX_STAGES) while
+// one stage still holds all the workers' bits; past that, two stages of the widest group that
+// fits. Returns the ring depth (0: does not fit), the total size, the offset of the second
+// weights and the bits per coordinate a stage holds.
 template <int QT>
-int ring_layout(int n, int smem_optin, size_t *smem_out, uint32_t *w2_offset)
+int ring_layout(int n, long long total_bits, int smem_optin, size_t *smem_out, uint32_t *w2_offset, uint32_t *group_bits)
 {
-    const size_t stage_bytes = size_t(QT) * 64 * AGC_DEC_GROUP_BITS;
     size_t tail = (2 * AGC_DEC_MAX_STAGES + 2) * sizeof(uint64_t) + sizeof(AgcDecWorker) * size_t(n) +
                   sizeof(int32_t) * (size_t(n) + 1) + 6 * size_t(n);
     tail = (tail + 15) & ~size_t(15);
     const size_t w2_rel = tail;
     tail += sizeof(float) * size_t(n) + 16;
     const size_t budget = size_t(smem_optin) - AGC_DEC_STATIC_SMEM;   // the kernel's static shared memory is set aside
-    if (budget < tail + 2 * stage_bytes) return 0;
-    long long stages = (long long)((budget - tail) / stage_bytes);
-    if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
+    if (budget < tail + 2 * size_t(QT) * 64 * 8) return 0;
+    const size_t per_bit = size_t(QT) * 64;
+    const long long want = total_bits < AGC_DEC_MAX_GROUP_BITS ? (total_bits < 8 ? 8 : total_bits) : AGC_DEC_MAX_GROUP_BITS;
+    int stages = 2;
+    long long bits = (long long)((budget - tail) / (2 * per_bit));
+    if (bits >= want) {
+        bits = want;
+        stages = (int)((budget - tail) / (per_bit * size_t(bits)));
+        if (stages > AGC_DEC_MAX_STAGES) stages = AGC_DEC_MAX_STAGES;
+    }
+    if (bits < 8) return 0;
+    const size_t stage_bytes = per_bit * size_t(bits);
     *smem_out = size_t(stages) * stage_bytes + tail;
     *w2_offset = uint32_t(size_t(stages) * stage_bytes + w2_rel);
-    return int(stages);
+    *group_bits = uint32_t(bits);
+    return stages;
 }
 
 template <int MODE, int QT>
@@ -1246,6 +1259,7 @@ int agc_launch_decode(agc_plan *plan, const void *codes, const float *scales, co
     P.status = status;
     P.stages = plan->dec_stages;
     P.w2_offset = plan->dec_w2_offset;
+    P.group_bits = plan->dec_group_bits;
     const bool collapsed = R > 1 && beta && !ghat;
     if (beta && R > 1) {
         if (cudaMemcpyAsync(plan->d_lr, lr_host, sizeof(float) * R, cudaMemcpyHostToDevice, stream) != cudaSuccess)
@@ -1344,8 +1358,12 @@ int agc_decode_prepare(agc_plan *plan, int smem_optin)
 {
     plan->dec_ring = false;
     if ((plan->flags & AGC_FLAG_FORCE_DIRECT) || plan->n > AGC_DEC_RING_MAX_WORKERS) return AGC_OK;
-    plan->dec_stages = ring_layout<AGC_DEC_QT>(plan->n, smem_optin, &plan->dec_smem, &plan->dec_w2_offset);
-    plan->dec2_stages = ring_layout<AGC_DEC_QT2>(plan->n, smem_optin, &plan->dec2_smem, &plan->dec2_w2_offset);
+    long long total_bits = 0;
+    for (int i = 0; i < plan->n; ++i) total_bits += plan->bits[i];
+    plan->dec_stages = ring_layout<AGC_DEC_QT>(plan->n, total_bits, smem_optin, &plan->dec_smem, &plan->dec_w2_offset,
+                                               &plan->dec_group_bits);
+    plan->dec2_stages = ring_layout<AGC_DEC_QT2>(plan->n, total_bits, smem_optin, &plan->dec2_smem, &plan->dec2_w2_offset,
+                                                 &plan->dec2_group_bits);
     if (plan->dec_stages < 2 || plan->dec2_stages < 2) return AGC_OK;
     // the limit is an attribute of the kernel, shared by all plans: the device's opt-in maximum
     const int ring_dyn = smem_optin - AGC_DEC_STATIC_SMEM;
@@ -1400,6 +1418,7 @@ int agc_launch_decode_two_track(agc_plan *plan, const void *codes, const float *
     P.status = status;
     P.stages = plan->dec2_stages;
     P.w2_offset = plan->dec2_w2_offset;
+    P.group_bits = plan->dec2_group_bits;
     P.v = plan->d_v;
     P.ghat_v = ghat_v;
     P.adam_m = m;

@@ -20,12 +20,10 @@
 #endif
 #define AGC_MAX_R 4096         // straggler realisations per decode call
 #ifndef AGC_DEC_QT
-#define AGC_DEC_QT 31          // pack blocks per decode tile = consumer warps of the ring decoder (+1 producer = 8 per scheduler)
+#define AGC_DEC_QT 23          // pack blocks per decode tile = consumer warps of the ring decoder (+1 producer = 6 per scheduler at 80 registers)
 #endif
-#ifndef AGC_DEC_GROUP_BITS
-#define AGC_DEC_GROUP_BITS 32  // cap on sum of b_i over a worker group: stage = QT * 64 * this bytes
-#endif
-#define AGC_DEC_MAX_STAGES 8
+#define AGC_DEC_MAX_STAGES 4
+#define AGC_DEC_MAX_GROUP_BITS 256  // 32 workers of 8 bits: the widest group a stage is ever sized for
 #define AGC_DEC_QT2 23         // consumer warps of the two-track decoder (two accumulator sets: 80 registers)
 #define AGC_DEC_MULTI_MIN_R 8    // from this many realisations on, g_hat of all of them comes from one pass over the messages
 #define AGC_DEC_RING_MAX_WORKERS 2048  // above this the per-worker tables no longer fit shared memory
@@ -108,6 +106,7 @@ struct AgcDecParams {
     int stages = 0;              // ring depth of the ring kernel
     int qt = 1;                  // blocks per tile of this ring launch (at most the kernel's QT)
     uint32_t w2_offset = 0;      // byte offset of the second-decoder array in shared memory
+    uint32_t group_bits = 0;     // cap on the sum of b_i over a worker group: a stage holds QT * 64 * group_bits bytes
     // residuals of many realisations
     const float *gref = nullptr;  // d reference values
     double *sqerr = nullptr;      // R sums of squared differences
@@ -147,6 +146,7 @@ struct agc_plan {
     int dec2_stages = 0;
     size_t dec2_smem = 0;
     uint32_t dec_w2_offset = 0, dec2_w2_offset = 0;
+    uint32_t dec_group_bits = 0, dec2_group_bits = 0;
     float *d_v = nullptr;
     // device tables
     int32_t *d_row_ptr = nullptr, *d_col_idx = nullptr;
