@@ -380,9 +380,6 @@ __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *
     weff[i] = s;
 }
 
-#ifndef AGC_DEC_PREFETCH
-#define AGC_DEC_PREFETCH 1
-#endif
 #ifndef AGC_DEC_LUT2
 #define AGC_DEC_LUT2 1
 #endif
@@ -712,11 +709,10 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
             const uint32_t nq = (uint32_t)(nblk - q0) < qt ? (uint32_t)(nblk - q0) : qt;
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int r0 = s_grp_ptr[g], nr = s_grp_ptr[g + 1] - r0;
-                uint32_t bytes = 0, soff = 0, wbits = 0;
+                uint32_t bytes = 0, soff = 0;
                 const unsigned char *src = nullptr;
                 if (lane < nr) {
                     const AgcDecWorker wk = s_wk[r0 + lane];
-                    wbits = wk.bits;
                     bytes = nq * 64u * wk.bits;
                     soff = wk.soff;
                     src = reinterpret_cast<const unsigned char *>(P.codes + wk.word_off + (long long)(q0 * 16 * (int)wk.bits));
@@ -730,15 +726,6 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
                 __syncwarp();
                 if (lane < nr) {
                     bulk_load_1d(smem + (size_t)s * stage_bytes + soff, src, bytes, &full[s]);
-#if AGC_DEC_PREFETCH
-                    // the same workers' chunks of this CTA's next tile row: on their way to L2 a
-                    // whole tile row ahead, so that the ring refills at L2 latency, not HBM latency
-                    const long long qn = q0 + (long long)gridDim.x * qt;
-                    if (qn < nblk) {
-                        const uint32_t nqn = (uint32_t)(nblk - qn) < qt ? (uint32_t)(nblk - qn) : qt;
-                        bulk_prefetch_l2(src + (size_t)gridDim.x * qt * 64u * wbits, nqn * 64u * wbits);
-                    }
-#endif
                 }
                 ++issued;
                 if (++s == stages) { s = 0; parity ^= 1u; }

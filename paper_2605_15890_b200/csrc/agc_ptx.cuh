@@ -90,11 +90,4 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
-// Ask for a range of global memory (16-byte aligned, a multiple of 16 bytes) to be brought
-// into L2; no completion is signalled and nothing is written.
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-
 }  // namespace
