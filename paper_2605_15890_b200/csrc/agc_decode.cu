@@ -744,7 +744,7 @@ __global__ void __launch_bounds__((QT + 1) * 32, 1) agc_decode_ring_kernel(const
         uint32_t parity = 0;
         bool ok = true;
         // scales of the lane's worker (lane < workers of the group) for this warp's block of a
-        // tile; fetched one tile ahead so that their latency hides behind the current tile
+        // tile; fetched one group ahead so that their latency hides behind the current group
         auto fetch_scales = [&](int T, int g, float (&sc)[4 / RB]) {   // T may lie one step past the last tile
 #pragma unroll
             for (int bk = 0; bk < 4 / RB; ++bk) sc[bk] = 0.0f;
