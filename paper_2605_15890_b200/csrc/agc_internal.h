@@ -47,7 +47,7 @@ struct __align__(8) AgcEntryDesc {
 };
 
 // One TMA box of a staged tile: partition rows [row, row + (32 >> hsel)) go to the
-// tile's row slots starting at `slot` (both 256-column halves).
+// tile's row slots starting at `slot` (512 columns each).
 struct AgcLoadOp {
     uint16_t slot;
     uint16_t hsel;
@@ -166,7 +166,7 @@ struct agc_plan {
     uint32_t *h_status = nullptr;
     void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled entry point
     // tensor maps of the last encode call (6 x 128 bytes, 64-byte aligned) and what they describe
-    alignas(64) unsigned char tmaps[AGC_ENC_BOX_SIZES * 128];
+    alignas(64) unsigned char tmaps[(AGC_ENC_BOX_SIZES + 1) * 128];
     const float *tmaps_G = nullptr;
     long long tmaps_ld = 0;
 };

@@ -207,7 +207,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     }
     for (int e = 0; e < nnz; ++e) {
         edesc[e].a = a[e];
-        edesc[e].off = stageable ? uint32_t(ent_slot[e]) * 1024u : 0u;
+        edesc[e].off = stageable ? uint32_t(ent_slot[e]) * 2048u : 0u;
     }
     pl->n_ops = int(ops.size());
     // tables of the staged encoder in shared memory: task records (32 bytes each), entry
@@ -216,7 +216,7 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
                                16 * size_t(pl->n_groups) + sizeof(AgcLoadOp) * ops.size() + 16;
     if (stageable && !(flags & AGC_FLAG_FORCE_DIRECT) && max_rows > 0 && table_bytes <= AGC_ENC_TABLE_BYTES_MAX) {
         const size_t tail = 2 * AGC_MAX_STAGES * sizeof(uint64_t) + 16 + table_bytes;
-        const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);  // two halves of max_rows x 1 KiB
+        const size_t stage_bytes = size_t(max_rows) * AGC_BLOCK * sizeof(float);  // max_rows x 2 KiB
         long long stages = (long long)((size_t(smem_optin) - tail - 1024) / stage_bytes);
         if (stages > AGC_MAX_STAGES) stages = AGC_MAX_STAGES;
         cudaDriverEntryPointQueryResult qres;
