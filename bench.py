@@ -32,9 +32,9 @@ FALLBACK_HBM_GBS = 6650.0
 # to d; valid for the cyclic cfg3 code with bucket 512 only, and only while the kernel is the
 # captured one):
 #   dram__bytes_read.sum + dram__bytes_write.sum per launch of the encode kernel
-NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 143.80}   # captured at d = 16,777,216 (messages larger than L2)
+NCU_TRAFFIC_BYTES_PER_COORD = {"cfg3": 143.82}   # captured at d = 16,777,216 (messages larger than L2)
 #   smsp__inst_executed.sum per (worker, pack block) task of the encode kernel
-NCU_WARP_INST_PER_TASK = {"cfg3": 306.5}
+NCU_WARP_INST_PER_TASK = {"cfg3": 307.4}
 
 
 def workload(name):
