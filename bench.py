@@ -87,15 +87,54 @@ def issue_rate(wl, bucket, code_kind, k1_ms, clocks):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons during a timed region."""
+    """SM clock, power and throttle reasons during a timed region: NVML polled from a thread about
+    every millisecond (the timed steps of the default run last some tens of milliseconds), or, where
+    NVML cannot be loaded, nvidia-smi every 50 ms."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"), (0x4, "sw_power_cap"))
 
     def __init__(self, index):
         self.index, self.lines, self.proc = index, [], None
+        self.nvml, self.handle, self.samples, self.stop_flag, self.th = None, None, [], False, None
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        handle = None
+        try:   # the CUDA device's own UUID: CUDA_VISIBLE_DEVICES may renumber the devices
+            import torch
+            uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+        except Exception:
+            handle = None
+        if handle is None:
+            handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        return pynvml, handle
+
+    def _poll(self):
+        nv, h = self.nvml, self.handle
+        reasons_fn = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self.stop_flag:
+            try:
+                self.samples.append((float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)),
+                                     nv.nvmlDeviceGetPowerUsage(h) / 1000.0, int(reasons_fn(h))))
+            except Exception:
+                break
+            time.sleep(0.001)
 
     def start(self):
+        try:
+            self.nvml, self.handle = self._nvml_handle()
+            self.smax = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.stop_flag = False
+            self.th = threading.Thread(target=self._poll, daemon=True)
+            self.th.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-lms", "50", "-i", str(self.index)],
@@ -106,14 +145,26 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        if self.proc is None:
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.th.join(timeout=5)
+            if self.samples:
+                sm = [x[0] for x in self.samples]
+                mask = 0
+                for x in self.samples:
+                    mask |= x[2]
+                return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": self.smax, "samples": len(sm),
+                        "reasons": sorted(name for bit, name in self.REASONS if mask & bit),
+                        "power_w_max": max(x[1] for x in self.samples), "source": "nvml"}
+        if self.proc is None and self.nvml is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        self.th.join(timeout=5)
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+            self.th.join(timeout=5)
         if not self.lines:
             # a region shorter than the sampling period: one reading taken right after it
             try:
@@ -139,7 +190,8 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons), "power_w_max": max(power) if power else None}
+                "samples": len(sm), "reasons": sorted(reasons), "power_w_max": max(power) if power else None,
+                "source": "nvidia-smi"}
 
 
 # ------------------------------------------------------------------ oracle legs (CPU)
