@@ -81,6 +81,7 @@ struct AgcEncParams {
     long long first_block;       // pack-block index of coordinate 0 in the random stream
     int n, k, n_groups, nnz, n_ops;
     int stages, stage_rows;
+    int split;                   // 1: CTA b stages the one tile (block b / n_groups, group b % n_groups)
     uint32_t round_lo, round_hi;
     uint32_t rk[20];             // Philox round keys: rk[2r] = key0 + r*W0, rk[2r+1] = key1 + r*W1
 };
@@ -136,6 +137,7 @@ struct agc_plan {
     // encode tiling
     bool use_tma = false;
     int n_groups = 0, stage_rows = 0, stages = 0, n_ops = 0;
+    bool enc_split = false;       // every (pack block, group) tile has a CTA of its own (few pack blocks)
     int rows_staged = 0;          // partition rows brought into shared memory per pack block, all groups together
     size_t enc_smem = 0;
     // decode ring

@@ -24,11 +24,11 @@ int upload(T **dst, const std::vector<T> &src)
 // Partition the workers (in order) into groups whose supports together touch at most
 // AGC_MAX_STAGE_ROWS partition rows: one staged tile = (pack block, group). Inside a tile
 // the rows sit in ascending partition order; each run of consecutive partitions is cut
-// into boxes of 32, 16, 8, 4, 2 or 1 rows. Returns false when some worker's own support
-// is too wide for a tile.
+// into boxes of 32, 16, 8, 4, 2 or 1 rows. A group holds at most max_workers workers.
+// Returns false when some worker's own support is too wide for a tile.
 bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::vector<int32_t> &grp_op_ptr,
                   std::vector<AgcLoadOp> &ops, std::vector<int32_t> &grp_wk_ptr,
-                  std::vector<int32_t> &grp_workers, std::vector<uint16_t> &ent_slot, int *max_rows)
+                  std::vector<int32_t> &grp_workers, std::vector<uint16_t> &ent_slot, int *max_rows, int max_workers)
 {
     grp_row_ptr.assign(1, 0);
     grp_op_ptr.assign(1, 0);
@@ -91,7 +91,8 @@ bool build_groups(const agc_plan &pl, std::vector<int32_t> &grp_row_ptr, std::ve
                 if (f < best_fresh) { best = i; best_fresh = f; }
             }
         }
-        if (int(cur_rows.size()) + best_fresh > AGC_MAX_STAGE_ROWS) {
+        if (int(cur_rows.size()) + best_fresh > AGC_MAX_STAGE_ROWS ||
+            int(grp_workers.size()) - grp_wk_ptr.back() >= max_workers) {
             flush();
             best = first_free;          // a new group starts from the lowest free worker
         }
@@ -189,8 +190,21 @@ extern "C" int agc_plan_create(agc_plan_t **out, int n_workers, int k_parts, int
     std::vector<AgcLoadOp> ops;
     std::vector<uint16_t> ent_slot;
     int max_rows = 0;
-    bool stageable = build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows);
+    bool stageable = build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows, n_workers);
     pl->n_groups = int(grp_row_ptr.size()) - 1;
+    // A vector of few pack blocks leaves most SMs without a tile: cut the workers into more,
+    // smaller groups, as many as still give every (block, group) tile an SM of its own.
+    if (stageable && pl->nblk * pl->n_groups < pl->sm_count) {
+        const int want = int(pl->sm_count / pl->nblk);
+        for (int cap = (n_workers + want - 1) / want; cap < n_workers; ++cap) {
+            build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows, cap);
+            if ((long long)(grp_row_ptr.size() - 1) * pl->nblk <= pl->sm_count) break;
+            if (cap + 1 == n_workers)   // no finer cut fits: back to the widest groups
+                build_groups(*pl, grp_row_ptr, grp_op_ptr, ops, grp_wk_ptr, grp_workers, ent_slot, &max_rows, n_workers);
+        }
+        pl->n_groups = int(grp_row_ptr.size()) - 1;
+    }
+    pl->enc_split = stageable && pl->nblk * pl->n_groups <= pl->sm_count;
     pl->rows_staged = grp_row_ptr.empty() ? 0 : int(grp_row_ptr.back());
     pl->use_tma = false;
     std::vector<AgcWorkerDesc> wdesc(n_workers);
