@@ -386,6 +386,12 @@ __global__ void agc_effective_weights_kernel(const uint8_t *masks, const float *
 // static shared memory of the ring kernel: the table of 2-bit level pairs (128 bytes), padded
 // to the 1 KiB alignment of the dynamic part
 #define AGC_DEC_STATIC_SMEM 1024
+// of the 8 pairs of 2-bit codes in a lane's word, this many take their levels from the table, the
+// others from shift + logic operation + packed subtraction: the table loads alone keep the
+// shared-memory pipe busier than the arithmetic pipes (measured: 8 / 7 / 6 / 5 / 4 pairs from the
+// table: 0.137 / 0.135 / 0.130 / 0.133 / 0.136 ms on a cfg3 mask with 30 received workers). The
+// two-track decoder, with two fmas per level, keeps all 8 on the table (0.222 against 0.233 ms).
+#define AGC_DEC_LUT2_PAIRS 6
 // ------------------------------------------------------------------ ring kernel
 // Persistent CTAs. A tile is AGC_DEC_QT consecutive pack blocks of one group of received
 // workers: the producer warp brings each worker's chunk (its words of those blocks are
@@ -487,10 +493,17 @@ __device__ __forceinline__ void ring_add_worker(const uint32_t (&W)[LaneWords<BI
     if constexpr (BITS == 2) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            // table address: 8 * nibble j merged into the 128-byte aligned base by one logic operation
-            const uint32_t addr = and_or(j == 0 ? A[0] << 3 : A[0] >> (4 * j - 3), 0x78u, lut2);
             float2 level;
-            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(level.x), "=f"(level.y) : "r"(addr));
+            if (j < (TWO ? 8 : AGC_DEC_LUT2_PAIRS)) {
+                // table address: 8 * nibble j merged into the 128-byte aligned base by one logic operation
+                const uint32_t addr = and_or(j == 0 ? A[0] << 3 : A[0] >> (4 * j - 3), 0x78u, lut2);
+                asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(level.x), "=f"(level.y) : "r"(addr));
+            } else {
+                // 2^23 + code by OR into the mantissa, then minus (2^23 + 1): exact
+                const uint32_t x0 = and_or(A[0] >> (4 * j), 3u, 0x4B000000u);
+                const uint32_t x1 = and_or(A[0] >> (4 * j + 2), 3u, 0x4B000000u);
+                level = __fadd2_rn(make_float2(__uint_as_float(x0), __uint_as_float(x1)), make_float2(-8388609.0f, -8388609.0f));
+            }
             const float c = cstep_row[j >> 1];
             const float2 r = __ffma2_rn(make_float2(c, c), level, make_float2(acc[2 * j], acc[2 * j + 1]));
             acc[2 * j] = r.x;
